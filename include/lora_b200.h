@@ -1,0 +1,230 @@
+/*
+ * lora_b200 -- unmerged multi-adapter LoRA forward for NVIDIA B200 (sm_100a).
+ *
+ *     y[t, :] = y_base[t, :] + s_i * (x[t, :] . A_i) . B_i ,      i = slot_idx[t]
+ *
+ * A LoRA adapter is a pair of low-rank matrices per adapted projection whose
+ * activations are added to the output of the backbone projection (paper
+ * Section 2.2).  Serving systems keep the adapters unmerged so that hundreds of
+ * them share one backbone, run several of them inside one batch, hold them in a
+ * statically reserved GPU region of A_max slots with one uniform footprint
+ * S_max each, and swap missing ones in from CPU memory (paper Sections 1, 2.2
+ * and the adapter-cache / Lat_load stage of Section 5, Eq. 1).  This library is
+ * that per-projection computation and the slot pool around it:
+ *
+ *   lora_pool_create      the A_max x S_max slot pool in caller-owned device memory
+ *   lora_pool_load_slot   side-stream swap-in of one adapter from pinned host memory
+ *   lora_build_segments   integer metadata: tokens grouped by adapter slot, cut in tiles
+ *   lora_bgmv_apply       decode batches (one token per request)
+ *   lora_sgmv_apply       prefill / chunked-prefill batches (per-adapter segments)
+ *
+ * Conventions
+ *  - plain C ABI; every call returns a lora_status_t; nothing aborts, traps or resets a device;
+ *  - "dev" pointers are device memory, "host" pointers are host memory; all buffers are owned
+ *    by the caller and must stay valid until the work queued on the stream has finished;
+ *  - streams are cudaStream_t values passed as void*; all GPU work is asynchronous on the
+ *    stream given; the library never synchronises a device and never allocates device memory;
+ *  - bf16 tensors are row-major with a leading dimension in ELEMENTS; base pointers must be
+ *    16-byte aligned and every d_in, d_out and leading dimension a multiple of 8;
+ *  - arithmetic: bf16 inputs, fp32 accumulation, one round-to-nearest-even to bf16 at the store.
+ */
+#ifndef LORA_B200_H
+#define LORA_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LORA_OK = 0,
+    LORA_ERR_INVALID_ARG = 1,      /* null pointer, bad enum, misaligned or overlapping buffers */
+    LORA_ERR_SHAPE = 2,            /* dimension not a multiple of 8, negative sizes */
+    LORA_ERR_SLOT_RANGE = 3,       /* slot >= num_slots or < 0 */
+    LORA_ERR_RANK = 4,             /* rank < 1 or rank > r_max */
+    LORA_ERR_NOT_LOADED = 5,       /* operation needs an occupied slot */
+    LORA_ERR_BUSY = 6,             /* reserved for hazards the host can see */
+    LORA_ERR_BUFFER_TOO_SMALL = 7, /* caller buffer smaller than the matching *_bytes query */
+    LORA_ERR_NOT_PINNED = 8,       /* host adapter memory is pageable */
+    LORA_ERR_CUDA = 9,             /* a CUDA runtime call failed: see lora_last_cuda_error() */
+    LORA_ERR_TIMEOUT = 10          /* a bounded device-side wait expired (device status word) */
+} lora_status_t;
+
+const char *lora_status_string(lora_status_t s);
+/* cudaError_t value of the most recent failing runtime call made by this thread's last call. */
+int32_t lora_last_cuda_error(void);
+/* Number of kernels this library has launched since it was loaded (all pools, all threads). */
+int64_t lora_launch_count(void);
+
+/* ----------------------------------------------------------------------------------------
+ * Slot pool (paper Section 2.2: a fixed region for adapter weights, at most A_max adapters
+ * loaded at once, every adapter given the same maximum footprint S_max).
+ * num_slots = A_max; r_max = the rank that S_max is sized for.
+ * -------------------------------------------------------------------------------------- */
+typedef struct lora_pool lora_pool_t;
+
+typedef struct {
+    int32_t d_in;    /* input width of the adapted projection  (multiple of 8) */
+    int32_t d_out;   /* output width of the adapted projection (multiple of 8) */
+} lora_target_t;
+
+typedef struct {
+    int32_t device;               /* CUDA device ordinal the pool lives on */
+    int32_t num_slots;            /* A_max, 1 .. 8192 */
+    int32_t r_max;                /* largest rank a slot can hold, 1 .. 64 */
+    int32_t num_targets;          /* adapted projections (e.g. 7 per layer x 32 layers) */
+    const lora_target_t *targets; /* host, [num_targets]; copied */
+    void *device_buf;             /* dev, 256-byte aligned, >= lora_pool_bytes(); caller-owned */
+    size_t device_buf_bytes;
+} lora_pool_desc_t;
+
+/* Bytes of device memory a pool of this shape needs (control block + transpose staging +
+ * num_slots slots of r_max rows for every target's A and B).  device_buf is ignored. */
+lora_status_t lora_pool_bytes(const lora_pool_desc_t *desc, size_t *bytes);
+
+/* Creates the host handle and clears the pool's control block (slot table: all slots empty;
+ * status words: zero).  Synchronous: returns after the clear has completed.  The handle is
+ * owned by the library; the device memory stays the caller's and must outlive the handle. */
+lora_status_t lora_pool_create(const lora_pool_desc_t *desc, lora_pool_t **out);
+lora_status_t lora_pool_destroy(lora_pool_t *pool);
+
+enum { LORA_A_DIN_MAJOR = 0,   /* A given as [d_in, rank] row-major (the formula's orientation) */
+       LORA_A_RANK_MAJOR = 1   /* A given as [rank, d_in] row-major (already in slot layout)    */ };
+
+typedef struct {
+    int32_t rank;            /* 1 .. r_max */
+    float scale;             /* s_i */
+    const void *const *A;    /* host, [num_targets] pointers to pinned bf16 matrices, see a_layout */
+    const void *const *B;    /* host, [num_targets] pointers to pinned bf16 [rank, d_out] row-major */
+    int32_t a_layout;        /* LORA_A_DIN_MAJOR or LORA_A_RANK_MAJOR */
+    int32_t trust_pinned;    /* non-zero: skip the per-pointer pinned-memory check */
+} lora_adapter_host_t;
+
+/*
+ * Swap one adapter into a slot (paper Section 5: the adapter-cache stage loads missing
+ * adapters from CPU memory; its cost is Lat_load in Eq. 1).  Queues on load_stream:
+ *   wait until everything queued so far on compute_stream has finished (the slot may still be
+ *   read), mark the slot empty, copy A and B for every target, zero the padding rows
+ *   rank .. r_max - 1, mark the slot occupied with (rank, scale), record the slot's ready event.
+ * Inside a slot every matrix is stored rank-major: A as [r_max, d_in], B as [r_max, d_out],
+ * rows 0 .. rank-1 meaningful, the rest zero.  LORA_A_DIN_MAJOR input is transposed on the device.
+ * Host matrices must stay valid until the ready event has fired (lora_pool_acquire + stream
+ * completion, or a synchronise on load_stream).  compute_stream may be NULL when no reader
+ * can be in flight.  On any error the slot is left untouched.
+ * Errors: INVALID_ARG, SLOT_RANGE, RANK, NOT_PINNED, CUDA.
+ */
+lora_status_t lora_pool_load_slot(lora_pool_t *pool, int32_t slot, const lora_adapter_host_t *adapter,
+                                  void *load_stream, void *compute_stream);
+
+/* Marks a slot empty (same ordering as a load: waits for compute_stream's queued readers). */
+lora_status_t lora_pool_evict_slot(lora_pool_t *pool, int32_t slot, void *load_stream,
+                                   void *compute_stream);
+
+/* Makes compute_stream wait for the ready events of these slots (host array of n slot ids).
+ * Slots that were never loaded are skipped.  Errors: SLOT_RANGE, CUDA. */
+lora_status_t lora_pool_acquire(lora_pool_t *pool, const int32_t *slots_host, int32_t n,
+                                void *compute_stream);
+
+/* Copies one slot's stored matrices of one target back to host memory (A_host: [r_max, d_in],
+ * B_host: [r_max, d_out], bf16) on `stream`; either pointer may be NULL.  For inspection. */
+lora_status_t lora_pool_read_slot(lora_pool_t *pool, int32_t slot, int32_t target,
+                                  void *A_host, void *B_host, void *stream);
+
+/* Host-side view of a slot as of the last load/evict call: rank (0 when empty) and scale. */
+lora_status_t lora_pool_slot_info(const lora_pool_t *pool, int32_t slot, int32_t *rank, float *scale);
+
+/* Device status words, copied asynchronously to host_out[4] (pinned host memory) on `stream`:
+ * [0] tokens whose slot id was neither -1 nor an occupied slot (accumulated; such tokens are
+ * treated as -1), [1] expired device-side waits, [2..3] reserved. */
+lora_status_t lora_pool_poll_status(lora_pool_t *pool, int32_t *host_out, void *stream);
+lora_status_t lora_pool_reset_status(lora_pool_t *pool, void *stream);
+
+/* Tuning knobs, for measurement.  key 0: apply algorithm (0 = default); see the library's
+ * documentation for the values.  Unknown keys -> INVALID_ARG. */
+lora_status_t lora_pool_set_tuning(lora_pool_t *pool, int32_t key, int32_t value);
+
+/* ----------------------------------------------------------------------------------------
+ * Segment metadata (several adapters are served inside one batch, paper Section 2.2; each
+ * request names its adapter, Section 5): a stable group-by-slot of the batch's tokens.
+ *
+ * Output buffer `meta_dev`, all int32, in this order (N = num_slots,
+ * cap_seg = min(T, N), cap_tile = cap_seg + T / tile_m):
+ *   header[16]   {T, n_active, n_invalid, n_seg, n_tile, tile_m, long_min, N, cap_seg, cap_tile, 0..}
+ *   perm[T]      active tokens ordered by (slot, token id), then the other tokens ascending
+ *   seg_slot[cap_seg], seg_start[cap_seg + 1], seg_rank[cap_seg], seg_flags[cap_seg]
+ *                flags bit0: the segment's tokens are consecutive ids; bit1: length >= long_min
+ *   tile_seg[cap_tile], tile_row0[cap_tile], tile_rows[cap_tile]
+ *                each segment cut into pieces of at most tile_m rows (positions in perm)
+ *   tile_flags[cap_tile]   bit0: the tile's tokens are consecutive ids
+ * Unused entries are -1.  A token is active iff its slot id names an occupied slot; a token
+ * that is neither active nor -1 is invalid (counted in header and in the pool's status word 0).
+ * The result is an exact integer function of its inputs.
+ * -------------------------------------------------------------------------------------- */
+lora_status_t lora_segments_bytes(int32_t T, int32_t num_slots, int32_t tile_m, size_t *bytes);
+
+/* slot_idx_dev: dev int32 [T]; meta_dev: dev, 16-byte aligned, meta_bytes >= lora_segments_bytes.
+ * tile_m in 1 .. 128, long_min >= 1.  T == 0 writes an empty table.  Uses the slot table as it is
+ * on the device when the kernel runs.  Errors: INVALID_ARG, SHAPE, BUFFER_TOO_SMALL, CUDA. */
+lora_status_t lora_build_segments(lora_pool_t *pool, const int32_t *slot_idx_dev, int32_t T,
+                                  int32_t tile_m, int32_t long_min,
+                                  void *meta_dev, size_t meta_bytes, void *stream);
+
+/* ----------------------------------------------------------------------------------------
+ * The forward itself.  x: bf16 [T, d_in]; y_base: bf16 [T, d_out] (the backbone projection's
+ * output, computed by the caller); y: bf16 [T, d_out], either exactly y_base (in place) or
+ * not overlapping it.  Tokens without an active slot get y = y_base bit for bit.  Row t of y
+ * depends only on row t of x and y_base, the token's slot and the pool.
+ * workspace: dev scratch of >= lora_workspace_bytes(pool, T) bytes (fp32 partial products
+ * v = x . A_i between the two phases), contents undefined afterwards; calls sharing a workspace
+ * must be ordered on one stream.
+ * T == 0 returns LORA_OK without launching.
+ * Errors: INVALID_ARG, SHAPE, SLOT_RANGE (target), BUFFER_TOO_SMALL, CUDA.
+ * -------------------------------------------------------------------------------------- */
+lora_status_t lora_workspace_bytes(const lora_pool_t *pool, int32_t T_max, size_t *bytes);
+
+/* Decode batches.  meta_dev_or_null: metadata built from the same slot_idx_dev (tile_m <= 16)
+ * so that each adapter's matrices are fetched once per group of tokens; NULL = index per token. */
+lora_status_t lora_bgmv_apply(lora_pool_t *pool, int32_t target,
+                              const void *x, int64_t ldx,
+                              const void *y_base, int64_t ldyb,
+                              void *y, int64_t ldy,
+                              const int32_t *slot_idx_dev, int32_t T,
+                              const void *meta_dev_or_null,
+                              void *workspace, size_t workspace_bytes, void *stream);
+
+/* Prefill / chunked-prefill batches.  meta_dev: metadata built for this batch (any tile_m).
+ * Full tiles of 128 consecutive tokens take the tensor-core path when the pool's tuning allows
+ * it; all other tiles take the CUDA-core path. */
+lora_status_t lora_sgmv_apply(lora_pool_t *pool, int32_t target,
+                              const void *x, int64_t ldx,
+                              const void *y_base, int64_t ldyb,
+                              void *y, int64_t ldy,
+                              const void *meta_dev, int32_t T,
+                              void *workspace, size_t workspace_bytes, void *stream);
+
+/* ----------------------------------------------------------------------------------------
+ * One layer step from HOST buffers: copies x, y_base and slot_idx (pinned host memory) to the
+ * caller's device staging buffers, builds the metadata, applies, and copies y back, all on
+ * `stream`.  kind: 0 = BGMV, 1 = SGMV.  y_host is complete when the stream has drained.
+ * -------------------------------------------------------------------------------------- */
+typedef struct {
+    void *x_dev;            /* >= T * d_in  bf16 */
+    void *y_base_dev;       /* >= T * d_out bf16 */
+    void *y_dev;            /* >= T * d_out bf16 (may equal y_base_dev) */
+    int32_t *slot_idx_dev;  /* >= T int32 */
+    void *meta_dev;         size_t meta_bytes;
+    void *workspace;        size_t workspace_bytes;
+} lora_step_buffers_t;
+
+lora_status_t lora_apply_host(lora_pool_t *pool, int32_t target, int32_t kind,
+                              const void *x_host, const void *y_base_host, void *y_host,
+                              const int32_t *slot_idx_host, int32_t T,
+                              int32_t tile_m, int32_t long_min,
+                              const lora_step_buffers_t *dev, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LORA_B200_H */

@@ -1,0 +1,177 @@
+// Shared declarations of the lora_b200 CUDA library (host handle, device views, metadata layout).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+#include <vector>
+
+#include "lora_b200.h"
+
+namespace lora {
+
+// ---------------------------------------------------------------------------------------------
+// error plumbing
+// ---------------------------------------------------------------------------------------------
+extern thread_local int32_t g_last_cuda_error;
+extern std::atomic<int64_t> g_launch_count;
+
+inline lora_status_t cuda_fail(cudaError_t e) {
+    g_last_cuda_error = (int32_t)e;
+    return LORA_ERR_CUDA;
+}
+#define LORA_CUDA_TRY(expr)                                   \
+    do {                                                      \
+        cudaError_t _e = (expr);                              \
+        if (_e != cudaSuccess) return ::lora::cuda_fail(_e);  \
+    } while (0)
+
+inline lora_status_t count_launch() {
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? LORA_OK : cuda_fail(e);
+}
+
+// ---------------------------------------------------------------------------------------------
+// device-side pool description
+// ---------------------------------------------------------------------------------------------
+struct SlotEntry {       // one per slot, in the pool's control block
+    int32_t rank;        // true rank, 0 when empty
+    float scale;         // s_i
+    int32_t loaded;      // 1 = occupied and complete
+    int32_t reserved;
+};
+
+enum { STATUS_INVALID_TOKENS = 0, STATUS_TIMEOUTS = 1, STATUS_WORDS = 4 };
+
+struct PoolView {                  // passed to kernels by value
+    const __nv_bfloat16 *weights;  // slot 0 of the weight region
+    int64_t slot_stride;           // elements between consecutive slots
+    const SlotEntry *table;        // [num_slots]
+    int32_t *status;               // [STATUS_WORDS]
+    int32_t num_slots;
+    int32_t r_max;
+};
+
+struct TargetView {    // one adapted projection inside a slot
+    int64_t off_a;     // element offset of A [r_max, d_in] inside a slot
+    int64_t off_b;     // element offset of B [r_max, d_out]
+    int32_t d_in;
+    int32_t d_out;
+};
+
+// ---------------------------------------------------------------------------------------------
+// segment metadata layout (int32 words)
+// ---------------------------------------------------------------------------------------------
+enum { META_HEADER_WORDS = 16 };
+enum { H_T = 0, H_NACTIVE = 1, H_NINVALID = 2, H_NSEG = 3, H_NTILE = 4, H_TILE_M = 5,
+       H_LONG_MIN = 6, H_NSLOTS = 7, H_CAP_SEG = 8, H_CAP_TILE = 9 };
+
+struct MetaLayout {
+    int32_t cap_seg, cap_tile;
+    int64_t perm, seg_slot, seg_start, seg_rank, seg_flags, tile_seg, tile_row0, tile_rows,
+        tile_flags, words;
+};
+
+__host__ __device__ inline MetaLayout meta_layout(int32_t T, int32_t num_slots, int32_t tile_m) {
+    MetaLayout L;
+    L.cap_seg = T < num_slots ? T : num_slots;
+    L.cap_tile = L.cap_seg + T / tile_m;
+    int64_t o = META_HEADER_WORDS;
+    L.perm = o;       o += T;
+    L.seg_slot = o;   o += L.cap_seg;
+    L.seg_start = o;  o += L.cap_seg + 1;
+    L.seg_rank = o;   o += L.cap_seg;
+    L.seg_flags = o;  o += L.cap_seg;
+    L.tile_seg = o;   o += L.cap_tile;
+    L.tile_row0 = o;  o += L.cap_tile;
+    L.tile_rows = o;  o += L.cap_tile;
+    L.tile_flags = o; o += L.cap_tile;
+    L.words = o;
+    return L;
+}
+
+// rank bucket a slot's kernels are specialised for: 8, 16, 32 or 64
+__host__ __device__ inline int32_t rank_bucket(int32_t r) {
+    return r <= 8 ? 8 : r <= 16 ? 16 : r <= 32 ? 32 : 64;
+}
+__host__ __device__ inline int32_t round_up8(int32_t r) { return (r + 7) & ~7; }
+
+}  // namespace lora
+
+// ---------------------------------------------------------------------------------------------
+// host handle
+// ---------------------------------------------------------------------------------------------
+struct lora_pool {
+    int32_t device = 0, num_slots = 0, r_max = 0, num_targets = 0;
+    std::vector<lora_target_t> targets;
+    std::vector<lora::TargetView> target_views;
+    char *base = nullptr;               // device_buf
+    size_t bytes = 0;
+    int32_t *status_dev = nullptr;      // [STATUS_WORDS]
+    lora::SlotEntry *table_dev = nullptr;
+    __nv_bfloat16 *staging_dev = nullptr;   // r_max * max_d_in elements, transpose input
+    size_t staging_elems = 0;
+    __nv_bfloat16 *weights_dev = nullptr;
+    int64_t slot_stride = 0;            // elements
+    std::vector<lora::SlotEntry> table_host;   // as of the last load / evict call
+    std::vector<cudaEvent_t> ready;     // per slot, created on first load
+    cudaEvent_t fence = nullptr;        // compute -> load ordering
+    int32_t sm_count = 148;
+    int32_t tuning[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+
+    // Shapes of the metadata tables built through this handle (the table itself lives on the
+    // device; apply calls need T and tile_m on the host to size their grids).
+    struct MetaRecord {
+        const void *ptr;
+        int32_t T, tile_m, long_min;
+    };
+    std::vector<MetaRecord> metas;
+    void remember_meta(const void *ptr, int32_t T, int32_t tile_m, int32_t long_min) {
+        for (MetaRecord &m : metas)
+            if (m.ptr == ptr) {
+                m.T = T; m.tile_m = tile_m; m.long_min = long_min;
+                return;
+            }
+        if (metas.size() >= 256) metas.erase(metas.begin());
+        metas.push_back({ptr, T, tile_m, long_min});
+    }
+    bool find_meta(const void *ptr, int32_t T, int32_t *tile_m) const {
+        for (const MetaRecord &m : metas)
+            if (m.ptr == ptr && m.T == T) {
+                *tile_m = m.tile_m;
+                return true;
+            }
+        return false;
+    }
+
+    lora::PoolView view() const {
+        lora::PoolView v;
+        v.weights = weights_dev;
+        v.slot_stride = slot_stride;
+        v.table = table_dev;
+        v.status = status_dev;
+        v.num_slots = num_slots;
+        v.r_max = r_max;
+        return v;
+    }
+};
+
+namespace lora {
+// RAII-free device guard: remembers the current device, switches, restores in the destructor.
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        want = dev;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0 && prev != want) cudaSetDevice(prev);
+    }
+    int want = -1;
+};
+}  // namespace lora

@@ -1,0 +1,205 @@
+// Segment metadata: a stable group-by-slot of the batch's tokens (several adapters are served
+// inside one batch, paper Section 2.2; each request names its adapter, Section 5), cut into row
+// tiles.  Integer work only; the result is a unique function of the inputs.
+//
+// One launch, no inter-block communication: every block recomputes the per-slot histogram and
+// its prefix sums (O(T + N) integer work from L2), then each warp owns whole slots and writes
+// that slot's run of `perm` by scanning the token list in order with warp ballots, which makes
+// the order inside a run ascending by construction.
+#include "common.cuh"
+
+namespace lora {
+
+constexpr int SEG_THREADS = 256;
+constexpr int SEG_WARPS = SEG_THREADS / 32;
+
+__device__ __forceinline__ bool token_active(const PoolView &pool, int32_t s) {
+    return s >= 0 && s < pool.num_slots && pool.table[s].loaded != 0;
+}
+
+__global__ void __launch_bounds__(SEG_THREADS)
+build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx, int32_t T,
+                      int32_t tile_m, int32_t long_min, int32_t *meta) {
+    extern __shared__ int32_t sm[];
+    const int32_t N = pool.num_slots;
+    int32_t *cnt = sm;             // [N] tokens per slot
+    int32_t *start = cnt + N;      // [N] first position in perm
+    int32_t *segid = start + N;    // [N] segment number
+    int32_t *tile0 = segid + N;    // [N] first tile number
+    __shared__ int32_t warp_tot[3][SEG_WARPS];
+    __shared__ int32_t totals[3];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const MetaLayout L = meta_layout(T, N, tile_m);
+
+    // ---- 1. histogram of active tokens ------------------------------------------------------
+    for (int32_t s = tid; s < N; s += SEG_THREADS) cnt[s] = 0;
+    __syncthreads();
+    for (int32_t t = tid; t < T; t += SEG_THREADS) {
+        const int32_t s = slot_idx[t];
+        if (token_active(pool, s)) atomicAdd(&cnt[s], 1);
+    }
+    __syncthreads();
+
+    // ---- 2. exclusive prefix sums over slots: positions, segment numbers, tile numbers ------
+    const int32_t per = (N + SEG_THREADS - 1) / SEG_THREADS;
+    const int32_t lo = min(tid * per, N), hi = min(lo + per, N);
+    int32_t c = 0, z = 0, tl = 0;
+    for (int32_t s = lo; s < hi; ++s) {
+        c += cnt[s];
+        z += cnt[s] > 0;
+        tl += (cnt[s] + tile_m - 1) / tile_m;
+    }
+    int32_t ic = c, iz = z, it = tl;   // inclusive warp scans
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int32_t a = __shfl_up_sync(0xffffffffu, ic, o);
+        const int32_t b = __shfl_up_sync(0xffffffffu, iz, o);
+        const int32_t d = __shfl_up_sync(0xffffffffu, it, o);
+        if (lane >= o) { ic += a; iz += b; it += d; }
+    }
+    if (lane == 31) { warp_tot[0][warp] = ic; warp_tot[1][warp] = iz; warp_tot[2][warp] = it; }
+    __syncthreads();
+    int32_t bc = 0, bz = 0, bt = 0;
+    for (int w = 0; w < warp; ++w) { bc += warp_tot[0][w]; bz += warp_tot[1][w]; bt += warp_tot[2][w]; }
+    int32_t rc = bc + ic - c, rz = bz + iz - z, rt = bt + it - tl;
+    for (int32_t s = lo; s < hi; ++s) {
+        start[s] = rc;
+        segid[s] = rz;
+        tile0[s] = rt;
+        rc += cnt[s];
+        rz += cnt[s] > 0;
+        rt += (cnt[s] + tile_m - 1) / tile_m;
+    }
+    if (tid == SEG_THREADS - 1) { totals[0] = rc; totals[1] = rz; totals[2] = rt; }
+    __syncthreads();
+    const int32_t n_active = totals[0], n_seg = totals[1], n_tile = totals[2];
+
+    int32_t *perm = meta + L.perm;
+    // ---- 3. one warp per occupied slot: write its run of perm, its segment and its tiles ----
+    for (int32_t s = blockIdx.x * SEG_WARPS + warp; s < N; s += gridDim.x * SEG_WARPS) {
+        const int32_t n = cnt[s];
+        if (n == 0) continue;
+        const int32_t p0 = start[s], seg = segid[s];
+        int32_t run = 0;
+        for (int32_t base = 0; base < T && run < n; base += 32) {
+            const int32_t t = base + lane;
+            const bool hit = t < T && slot_idx[t] == s;
+            const uint32_t m = __ballot_sync(0xffffffffu, hit);
+            if (hit) perm[p0 + run + __popc(m & ((1u << lane) - 1u))] = t;
+            run += __popc(m);
+        }
+        __syncwarp();
+        const int32_t first = perm[p0], last = perm[p0 + n - 1];
+        if (lane == 0) {
+            meta[L.seg_slot + seg] = s;
+            meta[L.seg_start + seg] = p0;
+            meta[L.seg_rank + seg] = pool.table[s].rank;
+            meta[L.seg_flags + seg] = (last - first + 1 == n ? 1 : 0) | (n >= long_min ? 2 : 0);
+        }
+        const int32_t nt = (n + tile_m - 1) / tile_m;
+        for (int32_t k = lane; k < nt; k += 32) {
+            const int32_t r0 = p0 + k * tile_m;
+            const int32_t rows = min(tile_m, p0 + n - r0);
+            const int32_t idx = tile0[s] + k;
+            meta[L.tile_seg + idx] = seg;
+            meta[L.tile_row0 + idx] = r0;
+            meta[L.tile_rows + idx] = rows;
+            meta[L.tile_flags + idx] = (perm[r0 + rows - 1] - perm[r0] + 1 == rows) ? 1 : 0;
+        }
+    }
+
+    // ---- 4. last block: header, the inactive tail of perm, -1 in unused entries -------------
+    if (blockIdx.x != gridDim.x - 1) return;
+    if (warp == 0) {
+        int32_t run = 0, n_invalid = 0;
+        for (int32_t base = 0; base < T; base += 32) {
+            const int32_t t = base + lane;
+            const int32_t s = t < T ? slot_idx[t] : -1;
+            const bool inact = t < T && !token_active(pool, s);
+            const uint32_t m = __ballot_sync(0xffffffffu, inact);
+            const uint32_t bad = __ballot_sync(0xffffffffu, inact && s != -1);
+            if (inact) perm[n_active + run + __popc(m & ((1u << lane) - 1u))] = t;
+            run += __popc(m);
+            n_invalid += __popc(bad);
+        }
+        if (lane == 0) {
+            meta[H_T] = T;
+            meta[H_NACTIVE] = n_active;
+            meta[H_NINVALID] = n_invalid;
+            meta[H_NSEG] = n_seg;
+            meta[H_NTILE] = n_tile;
+            meta[H_TILE_M] = tile_m;
+            meta[H_LONG_MIN] = long_min;
+            meta[H_NSLOTS] = N;
+            meta[H_CAP_SEG] = L.cap_seg;
+            meta[H_CAP_TILE] = L.cap_tile;
+            for (int i = H_CAP_TILE + 1; i < META_HEADER_WORDS; ++i) meta[i] = 0;
+            meta[L.seg_start + n_seg] = n_active;
+            if (n_invalid) atomicAdd(&pool.status[STATUS_INVALID_TOKENS], n_invalid);
+        }
+    } else {
+        const int t0 = tid - 32, nt = SEG_THREADS - 32;
+        for (int32_t i = n_seg + t0; i < L.cap_seg; i += nt) {
+            meta[L.seg_slot + i] = -1;
+            meta[L.seg_rank + i] = -1;
+            meta[L.seg_flags + i] = -1;
+        }
+        for (int32_t i = n_seg + 1 + t0; i <= L.cap_seg; i += nt) meta[L.seg_start + i] = -1;
+        for (int32_t i = n_tile + t0; i < L.cap_tile; i += nt) {
+            meta[L.tile_seg + i] = -1;
+            meta[L.tile_row0 + i] = -1;
+            meta[L.tile_rows + i] = -1;
+            meta[L.tile_flags + i] = -1;
+        }
+    }
+}
+
+lora_status_t launch_build_segments(lora_pool_t *pool, const int32_t *slot_idx_dev, int32_t T,
+                                    int32_t tile_m, int32_t long_min, void *meta_dev,
+                                    cudaStream_t stream) {
+    const int32_t N = pool->num_slots;
+    int grid = (N + SEG_WARPS - 1) / SEG_WARPS;
+    if (grid > 2 * pool->sm_count) grid = 2 * pool->sm_count;
+    if (grid < 1) grid = 1;
+    const size_t smem = sizeof(int32_t) * 4 * (size_t)N;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(build_segments_kernel,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    build_segments_kernel<<<grid, SEG_THREADS, smem, stream>>>(pool->view(), slot_idx_dev, T,
+                                                               tile_m, long_min, (int32_t *)meta_dev);
+    return count_launch();
+}
+
+}  // namespace lora
+
+using namespace lora;
+
+extern "C" {
+
+lora_status_t lora_segments_bytes(int32_t T, int32_t num_slots, int32_t tile_m, size_t *bytes) {
+    if (!bytes) return LORA_ERR_INVALID_ARG;
+    if (T < 0 || num_slots < 1 || tile_m < 1) return LORA_ERR_SHAPE;
+    *bytes = (size_t)meta_layout(T, num_slots, tile_m).words * sizeof(int32_t);
+    return LORA_OK;
+}
+
+lora_status_t lora_build_segments(lora_pool_t *pool, const int32_t *slot_idx_dev, int32_t T,
+                                  int32_t tile_m, int32_t long_min, void *meta_dev,
+                                  size_t meta_bytes, void *stream) {
+    if (!pool || !meta_dev || (T > 0 && !slot_idx_dev)) return LORA_ERR_INVALID_ARG;
+    if (T < 0 || tile_m < 1 || tile_m > 128 || long_min < 1) return LORA_ERR_SHAPE;
+    if ((uintptr_t)meta_dev & 15) return LORA_ERR_INVALID_ARG;
+    if (meta_bytes < (size_t)meta_layout(T, pool->num_slots, tile_m).words * sizeof(int32_t))
+        return LORA_ERR_BUFFER_TOO_SMALL;
+    DeviceGuard guard(pool->device);
+    if (!guard.ok) return cuda_fail(cudaErrorInvalidDevice);
+    lora_status_t s = launch_build_segments(pool, slot_idx_dev, T, tile_m, long_min, meta_dev,
+                                            (cudaStream_t)stream);
+    if (s == LORA_OK) pool->remember_meta(meta_dev, T, tile_m, long_min);
+    return s;
+}
+
+}  // extern "C"
