@@ -201,16 +201,10 @@ lora_status_t lora_pool_load_slot(lora_pool_t *pool, int32_t slot, const lora_ad
     set_slot_kernel<<<1, 32, 0, ls>>>(pool->table_dev, slot, 0, 0.0f, 0);
     if ((s = count_launch()) != LORA_OK) return s;
 
-    // gather the plain copies, merging neighbours that are adjacent on both sides
+    // One DMA per matrix.  Neighbouring host matrices are not merged into one copy: two pinned
+    // allocations can be adjacent in the address space, and a copy must not span both.
     std::vector<CopyJob> jobs;
     auto push = [&jobs](void *dst, const void *src, size_t bytes) {
-        if (!jobs.empty()) {
-            CopyJob &b = jobs.back();
-            if (b.dst + b.bytes == (char *)dst && b.src + b.bytes == (const char *)src) {
-                b.bytes += bytes;
-                return;
-            }
-        }
         jobs.push_back({(char *)dst, (const char *)src, bytes});
     };
     for (int32_t t = 0; t < pool->num_targets; ++t) {

@@ -138,8 +138,9 @@ class Workload:
         r = int(self.ranks[slot])
         rng = self._rng(1, slot, target)
         if self.weight_mode == "int":
-            A = rng.integers(-1, 2, size=(d_in, r)).astype(np.float32)
-            B = rng.integers(-2, 3, size=(r, d_out)).astype(np.float32)
+            # sparse small integers: every product and partial sum stays exactly representable
+            A = (rng.integers(-1, 2, size=(d_in, r)) * (rng.random((d_in, r)) < 0.25)).astype(np.float32)
+            B = (rng.integers(-1, 2, size=(r, d_out)) * (rng.random((r, d_out)) < 0.25)).astype(np.float32)
         else:
             lim = 1.0 / np.sqrt(d_in)
             A = rng.uniform(-lim, lim, size=(d_in, r)).astype(np.float32)
@@ -157,7 +158,7 @@ class Workload:
         T = self.T
         rng = self._rng(2, call)
         if self.act_mode == "int":
-            x = rng.integers(-1, 2, size=(T, d_in)).astype(np.float32)
+            x = (rng.integers(-1, 2, size=(T, d_in)) * (rng.random((T, d_in)) < 0.125)).astype(np.float32)
             yb = rng.integers(-8, 9, size=(T, d_out)).astype(np.float32)
         else:
             x = rng.standard_normal((T, d_in), dtype=np.float32)

@@ -144,7 +144,7 @@ def test_mixed_ranks_and_delta_isolation(grouped):
 def test_exact_integer_case_is_bit_exact(grouped, in_place):
     """Small-integer inputs: every intermediate is exact in fp32 and the result fits bf16, so
     the GPU must reproduce the oracle bit for bit."""
-    wl = W.make_custom(100, 256, 384, 9, [1, 4, 8, 16, 32], scale=2.0, weight_mode="int",
+    wl = W.make_custom(100, 2048, 1032, 9, [1, 4, 8, 16, 32], scale=2.0, weight_mode="int",
                        act_mode="int", frac_none=0.1)
     y_ref, _ = oracle_full(wl)
     assert np.abs(y_ref).max() < 256 and np.all(y_ref == np.rint(y_ref))
