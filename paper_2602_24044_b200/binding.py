@@ -298,4 +298,6 @@ def unpack_segments(meta: np.ndarray, T: int, num_slots: int, tile_m: int) -> Di
                     ("tile_row0", cap_tile), ("tile_rows", cap_tile), ("tile_flags", cap_tile)]:
         out[name] = meta[o:o + n].copy()
         o += n
+    o = (o + 3) & ~3
+    out["tile_desc"] = meta[o:o + 4 * cap_tile].reshape(cap_tile, 4).copy()   # library-private
     return out

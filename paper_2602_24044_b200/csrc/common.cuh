@@ -72,7 +72,7 @@ enum { H_T = 0, H_NACTIVE = 1, H_NINVALID = 2, H_NSEG = 3, H_NTILE = 4, H_TILE_M
 struct MetaLayout {
     int32_t cap_seg, cap_tile;
     int64_t perm, seg_slot, seg_start, seg_rank, seg_flags, tile_seg, tile_row0, tile_rows,
-        tile_flags, words;
+        tile_flags, tile_desc, words;
 };
 
 __host__ __device__ inline MetaLayout meta_layout(int32_t T, int32_t num_slots, int32_t tile_m) {
@@ -89,6 +89,8 @@ __host__ __device__ inline MetaLayout meta_layout(int32_t T, int32_t num_slots, 
     L.tile_row0 = o;  o += L.cap_tile;
     L.tile_rows = o;  o += L.cap_tile;
     L.tile_flags = o; o += L.cap_tile;
+    o = (o + 3) & ~(int64_t)3;            // library-private part, 16-byte aligned records
+    L.tile_desc = o;  o += 4 * (int64_t)L.cap_tile;   // {slot, row0, rows | rank << 16, scale bits}
     L.words = o;
     return L;
 }

@@ -106,6 +106,9 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx, int32
             meta[L.tile_row0 + idx] = r0;
             meta[L.tile_rows + idx] = rows;
             meta[L.tile_flags + idx] = (perm[r0 + rows - 1] - perm[r0] + 1 == rows) ? 1 : 0;
+            const SlotEntry e = pool.table[s];
+            *reinterpret_cast<int4 *>(meta + L.tile_desc + 4 * (int64_t)idx) =
+                make_int4(s, r0, rows | (e.rank << 16), __float_as_int(e.scale));
         }
     }
 

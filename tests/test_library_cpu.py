@@ -80,14 +80,17 @@ def test_segments_bytes_matches_documented_layout():
     T, N, tile_m = 256, 128, 16
     cap_seg, cap_tile = min(T, N), min(T, N) + T // tile_m
     words = 16 + T + 4 * cap_seg + 1 + 4 * cap_tile
+    public_words = words
+    words = (words + 3) // 4 * 4 + 4 * cap_tile          # library-private tile records
     assert lb.segments_bytes(T, N, tile_m) == 4 * words
-    assert lb.segments_bytes(0, N, tile_m) == 4 * 17
+    assert lb.segments_bytes(0, N, tile_m) == 4 * 20
     with pytest.raises(lb.LoraError):
         lb.segments_bytes(-1, N, tile_m)
     meta = np.arange(words, dtype=np.int32)
     parts = lb.unpack_segments(meta, T, N, tile_m)
     assert parts["perm"][0] == 16 and len(parts["tile_flags"]) == cap_tile
-    assert parts["tile_flags"][-1] == words - 1
+    assert parts["tile_flags"][-1] == public_words - 1
+    assert parts["tile_desc"][-1, -1] == words - 1
 
 
 def test_null_handles_are_rejected():
