@@ -195,6 +195,35 @@ lora_status_t lora_bgmv_apply(lora_pool_t *pool, int32_t target,
                               const void *meta_dev_or_null,
                               void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * lora_bgmv_apply for callers that cannot hand over a workspace (the paper has no counterpart;
+ * this is a convenience of the library).  Some hosts of this code may not allocate device
+ * memory at the point where they call it: a serving engine that has already given all free HBM
+ * to its KV cache and adapter pool, a plug-in running inside another framework's memory
+ * manager, code on a latency path where an allocation (or the implicit synchronisation of a
+ * free) is not acceptable.  For them the fp32 scratch between the shrink and expand phases is a
+ * fixed array of LORA_STATIC_SCRATCH_BYTES inside the library image; every GPU that loads the
+ * library holds that much memory until the process exits.
+ *  - Same arguments and results as lora_bgmv_apply minus the workspace; it always runs the
+ *    two-phase CUDA-core kernels.  It allocates and frees nothing.
+ *  - Limit: 32 * T * bucket(r_max) <= LORA_STATIC_SCRATCH_BYTES, bucket = r_max rounded up to
+ *    8, 16, 32 or 64 (T <= 4096 at r_max 16, T <= 1024 at r_max 64); beyond it the call returns
+ *    LORA_ERR_BUFFER_TOO_SMALL and launches nothing.
+ *  - The first call on each device looks up the array's device address; make that call before
+ *    starting any stream capture.
+ *  - All calls on a device share the one array, and it keeps whatever the last call left there
+ *    (the kernels overwrite every entry they later read, so nothing is cleared).  Two calls
+ *    that can overlap on the GPU (different streams without an ordering between them) race on
+ *    it: keep such calls on one stream or order them with events.
+ */
+#define LORA_STATIC_SCRATCH_BYTES (2u * 1024u * 1024u)
+lora_status_t lora_bgmv_apply_static(lora_pool_t *pool, int32_t target,
+                                     const void *x, int64_t ldx,
+                                     const void *y_base, int64_t ldyb,
+                                     void *y, int64_t ldy,
+                                     const int32_t *slot_idx_dev, int32_t T,
+                                     const void *meta_dev_or_null, void *stream);
+
 /* Prefill / chunked-prefill batches.  meta_dev: metadata built for this batch (any tile_m).
  * Full tiles of 128 consecutive tokens take the tensor-core path when the pool's tuning allows
  * it; all other tiles take the CUDA-core path. */

@@ -26,8 +26,9 @@ EXPORTS = [
     "lora_pool_evict_slot", "lora_pool_acquire", "lora_pool_read_slot", "lora_pool_slot_info",
     "lora_pool_poll_status", "lora_pool_reset_status", "lora_pool_set_tuning",
     "lora_segments_bytes", "lora_build_segments", "lora_workspace_bytes",
-    "lora_bgmv_apply", "lora_sgmv_apply", "lora_apply_host",
+    "lora_bgmv_apply", "lora_sgmv_apply", "lora_apply_host", "lora_bgmv_apply_static",
 ]
+STATIC_SCRATCH_BYTES = 2 * 1024 * 1024
 
 
 class LoraError(RuntimeError):
@@ -101,6 +102,7 @@ def _lib():
             "lora_workspace_bytes": [vp, i32, ctypes.POINTER(sz)],
             "lora_bgmv_apply": [vp, i32, vp, i64, vp, i64, vp, i64, vp, i32, vp, vp, sz, vp],
             "lora_sgmv_apply": [vp, i32, vp, i64, vp, i64, vp, i64, vp, i32, vp, sz, vp],
+            "lora_bgmv_apply_static": [vp, i32, vp, i64, vp, i64, vp, i64, vp, i32, vp, vp],
             "lora_apply_host": [vp, i32, i32, vp, vp, vp, vp, i32, i32, i32,
                                 ctypes.POINTER(_StepBuffers), vp],
         }
@@ -260,6 +262,16 @@ def bgmv_apply(pool: int, target: int, x, ldx: int, y_base, ldyb: int, y, ldy: i
     _check(_lib().lora_bgmv_apply(pool, int(target), _ptr(x), int(ldx), _ptr(y_base), int(ldyb),
                                   _ptr(y), int(ldy), _ptr(slot_idx_dev), int(T), _ptr(meta_dev),
                                   _ptr(workspace), nbytes, _stream(stream)), "lora_bgmv_apply")
+
+
+def bgmv_apply_static(pool: int, target: int, x, ldx: int, y_base, ldyb: int, y, ldy: int,
+                      slot_idx_dev, T: int, meta_dev, stream=None) -> None:
+    """lora_bgmv_apply without a workspace argument: the scratch is a fixed array inside the
+    library (for callers that must not allocate device memory).  See lora_b200.h for the size
+    limit and the rule about overlapping calls."""
+    _check(_lib().lora_bgmv_apply_static(pool, int(target), _ptr(x), int(ldx), _ptr(y_base),
+                                         int(ldyb), _ptr(y), int(ldy), _ptr(slot_idx_dev), int(T),
+                                         _ptr(meta_dev), _stream(stream)), "lora_bgmv_apply_static")
 
 
 def sgmv_apply(pool: int, target: int, x, ldx: int, y_base, ldyb: int, y, ldy: int, meta_dev,
