@@ -47,6 +47,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--algo", type=int, default=None,
+                    help="apply path: 0 fused cluster kernel (default), 1 two-phase kernels")
+    ap.add_argument("--cluster", type=int, default=None, help="fused path: cluster size 1/2/4/8")
     return ap.parse_args()
 
 
@@ -216,7 +219,12 @@ def main():
     wl = bench_workload()
     d_in, d_out = wl.targets[0]
     T = wl.T
-    s = Session(wl, device="cuda:%d" % local, a_layout=lb.A_RANK_MAJOR)
+    tuning = {}
+    if args.algo is not None:
+        tuning[0] = args.algo
+    if args.cluster is not None:
+        tuning[1] = args.cluster
+    s = Session(wl, device="cuda:%d" % local, a_layout=lb.A_RANK_MAJOR, tuning=tuning)
     dev = s.device
     xs, ybs, ys, metas = [], [], [], []
     meta_words = lb.segments_bytes(T, wl.num_slots, wl.tile_m) // 4
@@ -359,7 +367,9 @@ def main():
             "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
             "frac": achieved / peak, "peak_source": "%s copy bandwidth" % peak_kind,
             "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-            "kernel": "lora_bgmv_apply (shrink + expand)", "algorithmic_bytes_per_launch": alg,
+            "kernel": ("lora_bgmv_apply: shrink_kernel + expand_kernel (two launches)"
+                       if tuning.get(0) == 1 else "lora_bgmv_apply: fused_kernel (one launch)"),
+            "algorithmic_bytes_per_launch": alg,
             "us_per_launch": apply_ms * 1e3, "traffic": None,
         },
         "step_GBps": alg / (ms / K * 1e-3) / 1e9,

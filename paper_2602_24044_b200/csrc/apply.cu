@@ -62,7 +62,11 @@ static lora_status_t apply_common(lora_pool_t *pool, int32_t target, const void 
                                   cudaStream_t stream) {
     ApplyParams P;
     fill_apply_params(pool, P, target, x, ldx, yb, ldyb, y, ldy, slot_idx_dev, T, meta, tile_m);
-    return launch_twophase(pool, P, workspace, workspace_bytes, stream);
+    // the workspace contract holds on every path, whether or not the chosen kernels use it
+    if (!workspace || workspace_bytes < (size_t)T * P.RS * sizeof(float))
+        return LORA_ERR_BUFFER_TOO_SMALL;
+    if (pool->tuning[0] == 1) return launch_twophase(pool, P, workspace, workspace_bytes, stream);
+    return launch_fused(pool, P, stream);
 }
 }  // namespace lora
 

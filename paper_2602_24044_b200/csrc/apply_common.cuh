@@ -87,8 +87,8 @@ __device__ __forceinline__ Tile resolve_unit(const ApplyParams &P, const MetaLay
     t.valid = false;
     t.slot = -1; t.rank = 0; t.row0 = 0; t.rows = 0; t.scale = 0.0f;
     if (P.meta) {
-        if (u >= P.meta[H_NTILE]) return t;
         const int4 d = *reinterpret_cast<const int4 *>(P.meta + L.tile_desc + 4 * (int64_t)u);
+        if (d.x < 0) return t;   // unused entry
         t.slot = d.x;
         t.row0 = d.y;
         t.rows = d.z & 0xffff;

@@ -154,6 +154,7 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx, int32
             meta[L.tile_row0 + i] = -1;
             meta[L.tile_rows + i] = -1;
             meta[L.tile_flags + i] = -1;
+            *reinterpret_cast<int4 *>(meta + L.tile_desc + 4 * (int64_t)i) = make_int4(-1, 0, 0, 0);
         }
     }
 }

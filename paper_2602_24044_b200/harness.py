@@ -34,7 +34,7 @@ class Session:
 
     def __init__(self, wl, device: str = "cuda:0", targets: Optional[Sequence[int]] = None,
                  slots: Optional[Sequence[int]] = None, a_layout: int = lb.A_DIN_MAJOR,
-                 T_cap: Optional[int] = None):
+                 T_cap: Optional[int] = None, tuning: Optional[Dict[int, int]] = None):
         """targets: the workload's target ids to materialise in the pool (default: all);
         slots: which occupied slots to load (default: every slot the workload marks loaded)."""
         self.wl = wl
@@ -52,6 +52,8 @@ class Session:
         self.pool_mem = self.pool_buf[off:off + nbytes]
         self.pool = lb.pool_create(wl.num_slots, wl.r_max, self.pool_targets, self.pool_mem,
                                    self.dev_index)
+        for key, value in (tuning or {}).items():
+            lb.pool_set_tuning(self.pool, key, value)
         self.T_cap = int(T_cap if T_cap is not None else max(wl.T, 1))
         self.ws = torch.empty(lb.workspace_bytes(self.pool, self.T_cap), dtype=torch.uint8,
                               device=self.device)
