@@ -50,6 +50,7 @@ def parse_args():
     ap.add_argument("--algo", type=int, default=None,
                     help="apply path: 0 fused cluster kernel (default), 1 two-phase kernels")
     ap.add_argument("--cluster", type=int, default=None, help="fused path: cluster size 1/2/4/8")
+    ap.add_argument("--tile-m", type=int, default=None, help="rows per tile of the segment metadata")
     return ap.parse_args()
 
 
@@ -217,6 +218,8 @@ def main():
         dist.barrier()
 
     wl = bench_workload()
+    if args.tile_m is not None:
+        wl.tile_m = args.tile_m
     d_in, d_out = wl.targets[0]
     T = wl.T
     tuning = {}

@@ -25,7 +25,7 @@ struct ApplyParams {
     int32_t in_place;
     // fused path: shared-memory carve-up (bytes from the start of dynamic shared memory)
     int32_t rows_cap;          // rows a unit can have, rounded up to 16
-    int32_t off_part, off_vst, off_stage;
+    int32_t off_part, off_vst, off_stage, off_x;
     int32_t path_filter;       // 0 = every tile, 1 = skip tiles taken by the tensor-core kernel
 };
 
@@ -118,7 +118,8 @@ __device__ __forceinline__ void copy_rows(const ApplyParams &P, const int32_t *r
     for (int32_t m = 0; m < rows; ++m) {
         const __nv_bfloat16 *src = P.yb + (int64_t)rowidx[m] * P.ldyb;
         __nv_bfloat16 *dst = P.y + (int64_t)rowidx[m] * P.ldy;
-        for (int32_t v = part * AP_THREADS + threadIdx.x; v < vecs; v += parts * AP_THREADS)
+        for (int32_t v = part * (int32_t)blockDim.x + threadIdx.x; v < vecs;
+             v += parts * (int32_t)blockDim.x)
             reinterpret_cast<uint4 *>(dst)[v] = ldg16(src + (int64_t)v * 8);
     }
 }

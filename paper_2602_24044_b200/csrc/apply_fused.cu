@@ -3,18 +3,26 @@
 // A thread-block cluster owns one unit (a row tile of one adapter, or one token).  Block c of
 // the cluster takes the c-th slice of d_in for the shrink phase and the c-th slice of d_out for
 // the expand phase:
-//   1. all operands of both phases (A_i slice, x rows, B_i slice, y_base rows) are requested up
-//      front with bulk asynchronous copies into shared memory, each group signalled by an mbarrier;
-//      the expand operands do not depend on the shrink result, so their latency hides behind it;
-//   2. shrink: fp32 partial v over the block's d_in slice (split-K, warp-shuffle reduction);
+//   1. the weight slices of both phases (A_i, B_i) are requested up front with bulk asynchronous
+//      copies into shared memory, each signalled by an mbarrier; the y_base rows are prefetched
+//      into L2; none of this depends on the shrink result, so its latency hides behind it;
+//   2. shrink: fp32 partial v over the block's d_in slice (split-K, warp-shuffle reduction),
+//      x rows read straight from global memory with 128-bit loads;
 //   3. the partials are exchanged through distributed shared memory and summed in block order,
 //      identically in every block (no global workspace, no float atomics);
 //   4. expand over the block's d_out slice with the scale and the residual add fused, bf16 store.
+// Blocks are kept small (128 threads, only the weight slices staged) so that many are resident
+// per SM: a decode batch fits on the GPU in one wave and the hardware overlaps their latencies.
 // Every per-row sum is taken in a fixed order that does not depend on which other rows share the
 // tile, so a row's result depends only on its own inputs.
 #include "apply_common.cuh"
 
 namespace lora {
+
+constexpr int FT = 128;   // threads per block of the fused kernel
+#ifndef LORA_FUSED_MIN_BLOCKS
+#define LORA_FUSED_MIN_BLOCKS 5   // resident blocks per SM the register budget is held to
+#endif
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -58,6 +66,9 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t by
         "l"(src), "r"(bytes), "r"(smem_u32(bar))
         : "memory");
 }
+__device__ __forceinline__ void prefetch_l2(const void *p) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -83,36 +94,46 @@ __device__ __forceinline__ float ld_peer_f32(uint32_t local_addr, uint32_t rank)
     return v;
 }
 
-enum { BAR_A = 0, BAR_X = 1, BAR_B = 2, BAR_Y = 3 };
+enum { BAR_A = 0, BAR_B = 1, BAR_X = 2 };
+constexpr int XROWS = 16;                // x rows staged at a time
 constexpr int FUSED_HEAD_BYTES = 1024;   // mbarriers (64 B) + row indices (ROWS_CAP * 4 B)
 
-// One warp requests `nrows` rows of `ncols` bf16 each; row r comes from src(r) and lands at
-// stage + r * pitch.
-template <typename SrcFn>
+// One warp requests `nrows` rows of `ncols` bf16 each; row r comes from src + r * src_pitch and
+// lands at stage + r * pitch.
 __device__ __forceinline__ void issue_rows(uint64_t *bar, __nv_bfloat16 *stage, int pitch, int nrows,
-                                           int ncols, int lane, SrcFn src) {
+                                           int ncols, int lane, const __nv_bfloat16 *src,
+                                           int64_t src_pitch) {
     if (lane == 0) mbar_expect_tx(bar, (uint32_t)nrows * (uint32_t)ncols * 2u);
     __syncwarp();
-    for (int r = lane; r < nrows; r += 32) bulk_g2s(stage + r * pitch, src(r), (uint32_t)ncols * 2u, bar);
+    for (int r = lane; r < nrows; r += 32)
+        bulk_g2s(stage + r * pitch, src + (int64_t)r * src_pitch, (uint32_t)ncols * 2u, bar);
+}
+// the same for rows picked by an index list (token rows of a tile)
+__device__ __forceinline__ void issue_gather(uint64_t *bar, __nv_bfloat16 *stage, int pitch, int nrows,
+                                             int ncols, int lane, const __nv_bfloat16 *src,
+                                             int64_t src_pitch, const int32_t *idx) {
+    if (lane == 0) mbar_expect_tx(bar, (uint32_t)nrows * (uint32_t)ncols * 2u);
+    __syncwarp();
+    for (int r = lane; r < nrows; r += 32)
+        bulk_g2s(stage + r * pitch, src + (int64_t)idx[r] * src_pitch, (uint32_t)ncols * 2u, bar);
 }
 
-template <int RP, int KPT, int CVE>
+// RP: rank bucket; DCA / DCB: columns of A / B staged at a time.
+template <int RP, int DCA, int DCB>
 __device__ __forceinline__ void fused_body(const ApplyParams &P, const Tile &tl, unsigned char *smem,
                                            uint32_t crank, uint32_t csize) {
-    constexpr int KG = RP / KPT, CV = AP_THREADS / KG, DCA = CV * 8, WPK = CV / 32, MG = 32 / KPT;
-    constexpr int NMG = AP_THREADS / CVE, RPT = 16 / NMG, DCB = CVE * 8;
-    constexpr int A_BYTES = RP * DCA * 2, X_BYTES = 16 * DCA * 2, B_BYTES = RP * DCB * 2;
-    static_assert(MG <= 16 && RPT >= 1, "mapping");
+    constexpr int CV = DCA / 8, KG = FT / CV, KPT = RP / KG, MG = 32 / KPT, WPK = CV / 32;
+    constexpr int CVE = DCB / 8, NMG = FT / CVE, RPT = 4, EG = NMG * RPT;   // EG rows per expand pass
+    constexpr int A_BYTES = RP * DCA * 2;
+    static_assert(KPT * MG == 32 && WPK >= 1 && KG * KPT == RP, "shrink mapping");
 
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem);
     const int32_t *rowidx = reinterpret_cast<const int32_t *>(smem + 64);
     float *part = reinterpret_cast<float *>(smem + P.off_part);
     float *vsT = reinterpret_cast<float *>(smem + P.off_vst);
     __nv_bfloat16 *As = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_stage);
-    __nv_bfloat16 *Xs = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_stage + A_BYTES);
-    __nv_bfloat16 *Bs = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_stage + A_BYTES + X_BYTES);
-    __nv_bfloat16 *Ys =
-        reinterpret_cast<__nv_bfloat16 *>(smem + P.off_stage + A_BYTES + X_BYTES + B_BYTES);
+    __nv_bfloat16 *Bs = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_stage + A_BYTES);
+    __nv_bfloat16 *Xs = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_x);   // [XROWS][DCA]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t d_in = P.tv.d_in, d_out = P.tv.d_out, rows = tl.rows, rank = tl.rank;
@@ -127,93 +148,86 @@ __device__ __forceinline__ void fused_body(const ApplyParams &P, const Tile &tl,
     const int32_t Wb = (d_out + (int32_t)csize * 8 - 1) / ((int32_t)csize * 8) * 8;
     const int32_t b_lo = min((int32_t)crank * Wb, d_out), b_hi = min(b_lo + Wb, d_out);
     const int32_t nb = (b_hi - b_lo + DCB - 1) / DCB;
-    const int32_t nsub = (rows + 15) >> 4;
 
-    auto issue_A = [&](int32_t c) {
-        const int32_t col0 = a_lo + c * DCA, ncols = min(DCA, a_hi - col0);
-        issue_rows(&bars[BAR_A], As, DCA, rank, ncols, lane,
-                   [&](int r) { return A + (int64_t)r * d_in + col0; });
-    };
-    auto issue_X = [&](int32_t sub, int32_t c) {
-        const int32_t col0 = a_lo + c * DCA, ncols = min(DCA, a_hi - col0);
-        const int32_t m0 = sub * 16, nrows = min(16, rows - m0);
-        issue_rows(&bars[BAR_X], Xs, DCA, nrows, ncols, lane,
-                   [&](int r) { return P.x + (int64_t)rowidx[m0 + r] * P.ldx + col0; });
-    };
-    auto issue_B = [&](int32_t c) {
-        const int32_t col0 = b_lo + c * DCB, ncols = min(DCB, b_hi - col0);
-        issue_rows(&bars[BAR_B], Bs, DCB, rank, ncols, lane,
-                   [&](int r) { return B + (int64_t)r * d_out + col0; });
-    };
-    auto issue_Y = [&](int32_t sub, int32_t c) {
-        const int32_t col0 = b_lo + c * DCB, ncols = min(DCB, b_hi - col0);
-        const int32_t m0 = sub * 16, nrows = min(16, rows - m0);
-        issue_rows(&bars[BAR_Y], Ys, DCB, nrows, ncols, lane,
-                   [&](int r) { return P.yb + (int64_t)rowidx[m0 + r] * P.ldyb + col0; });
-    };
-
-    // first requests of both phases go out before any arithmetic
-    if (warp == 0 && na > 0) { issue_A(0); issue_X(0, 0); }
-    if (warp == 1 && nb > 0) { issue_B(0); issue_Y(0, 0); }
-    for (int i = tid; i < WPK * rows * RP; i += AP_THREADS) part[i] = 0.0f;
+    // weight slices of both phases go out before any arithmetic
+    if (warp == 0 && na > 0)
+        issue_rows(&bars[BAR_A], As, DCA, rank, min(DCA, a_hi - a_lo), lane, A + a_lo, d_in);
+    if (warp == 1 && nb > 0)
+        issue_rows(&bars[BAR_B], Bs, DCB, rank, min(DCB, b_hi - b_lo), lane, B + b_lo, d_out);
+    if (warp == 2 && na > 0)
+        issue_gather(&bars[BAR_X], Xs, DCA, min(XROWS, rows), min(DCA, a_hi - a_lo), lane,
+                     P.x + a_lo, P.ldx, rowidx);
+    // pull this block's y_base columns towards L2 (128-byte lines); they are needed last
+    if (b_hi > b_lo) {
+        const int32_t lines = ((b_hi - b_lo) * 2 + 127) >> 7;
+        for (int i = tid; i < rows * lines; i += FT) {
+            const int m = i / lines, l = i - m * lines;
+            prefetch_l2(reinterpret_cast<const char *>(P.yb + (int64_t)rowidx[m] * P.ldyb + b_lo) +
+                        (l << 7));
+        }
+    }
+    for (int i = tid; i < WPK * rows * RP; i += FT) part[i] = 0.0f;
     __syncthreads();
 
-    uint32_t ph_a = 0, ph_x = 0, ph_b = 0, ph_y = 0;
+    uint32_t ph_a = 0, ph_b = 0, ph_x = 0;
     bool ok = true;
 
-    // ---- shrink -------------------------------------------------------------------------------
+    // ---- shrink: thread = (column vector cv, rank group kg); KPT ranks x MG rows per reduction -
     {
         const int kg = tid / CV, cv = tid % CV, wk = cv >> 5;
         for (int32_t c = 0; c < na; ++c) {
-            const int32_t ncols = min(DCA, a_hi - (a_lo + c * DCA));
+            const int32_t col0 = a_lo + c * DCA, ncols = min(DCA, a_hi - col0);
             const bool cvalid = cv * 8 < ncols;
-            if (c > 0 && warp == 0) issue_A(c);
+            if (c > 0 && warp == 0)
+                issue_rows(&bars[BAR_A], As, DCA, rank, ncols, lane, A + col0, d_in);
             ok = mbar_wait(&bars[BAR_A], ph_a) && ok;
             ph_a ^= 1;
-            float a[KPT][8];
+            for (int32_t m0 = 0; m0 < rows; m0 += MG) {
+                if ((m0 % XROWS) == 0) {
+                    // next XROWS rows of x: requested here unless it is the very first group,
+                    // whose request went out at the start
+                    if (c > 0 || m0 > 0) {
+                        __syncthreads();   // everyone is done with the previous rows
+                        if (warp == 2)
+                            issue_gather(&bars[BAR_X], Xs, DCA, min(XROWS, rows - m0), ncols, lane,
+                                         P.x + col0, P.ldx, rowidx + m0);
+                    }
+                    ok = mbar_wait(&bars[BAR_X], ph_x) && ok;
+                    ph_x ^= 1;
+                }
+                float xf[MG][8];
 #pragma unroll
-            for (int kk = 0; kk < KPT; ++kk) {
-                const int k = kg * KPT + kk;
-                uint4 w = make_uint4(0, 0, 0, 0);
-                if (cvalid && k < rank) w = *reinterpret_cast<const uint4 *>(As + k * DCA + cv * 8);
-                unpack8(w, a[kk]);
-            }
-            for (int32_t sub = 0; sub < nsub; ++sub) {
-                if ((c > 0 || sub > 0) && warp == 0) issue_X(sub, c);
-                ok = mbar_wait(&bars[BAR_X], ph_x) && ok;
-                ph_x ^= 1;
-                const int32_t m0 = sub * 16, nrows = min(16, rows - m0);
+                for (int mi = 0; mi < MG; ++mi) {
+                    uint4 xv = make_uint4(0, 0, 0, 0);
+                    if (cvalid && m0 + mi < rows)
+                        xv = *reinterpret_cast<const uint4 *>(Xs + ((m0 % XROWS) + mi) * DCA + cv * 8);
+                    unpack8(xv, xf[mi]);
+                }
+                float acc[32];
 #pragma unroll
-                for (int g = 0; g < 16; g += MG) {
-                    if (g < nrows) {
-                        float acc[32];
+                for (int kk = 0; kk < KPT; ++kk) {
+                    const int k = kg * KPT + kk;
+                    uint4 w = make_uint4(0, 0, 0, 0);
+                    if (cvalid && k < rank) w = *reinterpret_cast<const uint4 *>(As + k * DCA + cv * 8);
+                    float af[8];
+                    unpack8(w, af);
 #pragma unroll
-                        for (int mi = 0; mi < MG; ++mi) {
-                            uint4 xv = make_uint4(0, 0, 0, 0);
-                            if (cvalid && g + mi < nrows)
-                                xv = *reinterpret_cast<const uint4 *>(Xs + (g + mi) * DCA + cv * 8);
-                            float xf[8];
-                            unpack8(xv, xf);
+                    for (int mi = 0; mi < MG; ++mi) {
+                        float s = 0.0f;
 #pragma unroll
-                            for (int kk = 0; kk < KPT; ++kk) {
-                                float s = 0.0f;
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) s = fmaf(xf[e], a[kk][e], s);
-                                acc[mi * KPT + kk] = s;
-                            }
-                        }
-                        const float tot = warp_reduce32(acc, lane);
-                        const int mi = lane / KPT, kk = lane % KPT;
-                        if (g + mi < nrows)
-                            part[(wk * rows + m0 + g + mi) * RP + kg * KPT + kk] += tot;
+                        for (int e = 0; e < 8; ++e) s = fmaf(xf[mi][e], af[e], s);
+                        acc[mi * KPT + kk] = s;
                     }
                 }
-                __syncthreads();   // the x stage (and after the last sub-tile the A stage) is free
+                const float tot = warp_reduce32(acc, lane);
+                const int mi = lane / KPT, kk = lane % KPT;
+                if (m0 + mi < rows) part[(wk * rows + m0 + mi) * RP + kg * KPT + kk] += tot;
             }
+            __syncthreads();   // the A stage is free
         }
     }
     if (WPK > 1) {
-        for (int i = tid; i < rows * RP; i += AP_THREADS) {
+        for (int i = tid; i < rows * RP; i += FT) {
             float v = part[i];
 #pragma unroll
             for (int w = 1; w < WPK; ++w) v += part[w * rows * RP + i];
@@ -225,9 +239,9 @@ __device__ __forceinline__ void fused_body(const ApplyParams &P, const Tile &tl,
     cluster_wait();
     {
         const uint32_t part_addr = smem_u32(part);
-        const int32_t rows16 = (rows + 15) & ~15;
-        for (int i = tid; i < rows16 * rank; i += AP_THREADS) {
-            const int m = i / rank, k = i % rank;
+        const int32_t rows_pad = (rows + EG - 1) / EG * EG;
+        for (int i = tid; i < rows_pad * rank; i += FT) {
+            const int m = i / rank, k = i - m * rank;
             float v = 0.0f;
             if (m < rows)
                 for (uint32_t q = 0; q < csize; ++q)
@@ -238,23 +252,27 @@ __device__ __forceinline__ void fused_body(const ApplyParams &P, const Tile &tl,
     cluster_arrive();   // done reading the peers; the matching wait is at the end
     __syncthreads();
 
-    // ---- expand -------------------------------------------------------------------------------
+    // ---- expand: thread = (output column vector jv, row group mg), RPT rows at a time ----------
     {
         const int mg = tid / CVE, jv = tid % CVE;
         const float s = tl.scale;
         for (int32_t c = 0; c < nb; ++c) {
             const int32_t col0 = b_lo + c * DCB, ncols = min(DCB, b_hi - col0);
             const bool cvalid = jv * 8 < ncols;
-            if (c > 0 && warp == 1) issue_B(c);
+            if (c > 0 && warp == 1)
+                issue_rows(&bars[BAR_B], Bs, DCB, rank, ncols, lane, B + col0, d_out);
             ok = mbar_wait(&bars[BAR_B], ph_b) && ok;
             ph_b ^= 1;
-            for (int32_t sub = 0; sub < nsub; ++sub) {
-                if ((c > 0 || sub > 0) && warp == 1) issue_Y(sub, c);
-                ok = mbar_wait(&bars[BAR_Y], ph_y) && ok;
-                ph_y ^= 1;
-                const int32_t m0 = sub * 16, nrows = min(16, rows - m0);
-                const int32_t ml = mg * RPT;   // first local row of this thread
-                if (cvalid && ml < nrows) {
+            for (int32_t m0 = 0; m0 < rows; m0 += EG) {
+                const int32_t mb = m0 + mg * RPT;
+                if (cvalid && mb < rows) {
+                    uint4 ybv[RPT];
+#pragma unroll
+                    for (int i = 0; i < RPT; ++i) {
+                        ybv[i] = make_uint4(0, 0, 0, 0);
+                        if (mb + i < rows)
+                            ybv[i] = ldg16(P.yb + (int64_t)rowidx[mb + i] * P.ldyb + col0 + jv * 8);
+                    }
                     float acc[RPT][8];
 #pragma unroll
                     for (int i = 0; i < RPT; ++i)
@@ -264,16 +282,8 @@ __device__ __forceinline__ void fused_body(const ApplyParams &P, const Tile &tl,
                     for (int32_t k = 0; k < rank; ++k) {
                         float bf[8];
                         unpack8(*reinterpret_cast<const uint4 *>(Bs + k * DCB + jv * 8), bf);
-                        float vv[RPT];
-                        if (RPT == 4) {
-                            const float4 v4 =
-                                *reinterpret_cast<const float4 *>(vsT + k * VSP + m0 + ml);
-                            vv[0] = v4.x; vv[1] = v4.y; vv[2 % RPT] = v4.z; vv[3 % RPT] = v4.w;
-                        } else {
-                            const float2 v2 =
-                                *reinterpret_cast<const float2 *>(vsT + k * VSP + m0 + ml);
-                            vv[0] = v2.x; vv[1 % RPT] = v2.y;
-                        }
+                        const float4 v4 = *reinterpret_cast<const float4 *>(vsT + k * VSP + mb);
+                        const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
 #pragma unroll
                         for (int i = 0; i < RPT; ++i)
 #pragma unroll
@@ -281,25 +291,21 @@ __device__ __forceinline__ void fused_body(const ApplyParams &P, const Tile &tl,
                     }
                     if (ok) {
 #pragma unroll
-                        for (int i = 0; i < RPT; ++i) {
-                            if (ml + i < nrows) {
-                                const uint4 ybv =
-                                    *reinterpret_cast<const uint4 *>(Ys + (ml + i) * DCB + jv * 8);
-                                *reinterpret_cast<uint4 *>(P.y + (int64_t)rowidx[m0 + ml + i] * P.ldy +
-                                                           col0 + jv * 8) = finish8(acc[i], ybv, s);
-                            }
-                        }
+                        for (int i = 0; i < RPT; ++i)
+                            if (mb + i < rows)
+                                *reinterpret_cast<uint4 *>(P.y + (int64_t)rowidx[mb + i] * P.ldy + col0 +
+                                                           jv * 8) = finish8(acc[i], ybv[i], s);
                     }
                 }
-                __syncthreads();   // the y_base stage (and after the last sub-tile the B stage) is free
             }
+            __syncthreads();   // the B stage is free
         }
     }
     if (!ok && tid == 0) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
     cluster_wait();   // no block leaves while a peer may still read its partials
 }
 
-__global__ void __launch_bounds__(AP_THREADS, 2)
+__global__ void __launch_bounds__(FT, LORA_FUSED_MIN_BLOCKS)
 fused_kernel(const ApplyParams P) {
     extern __shared__ __align__(128) unsigned char smem[];
     const uint32_t csize = cluster_nctarank(), crank = cluster_ctarank();
@@ -321,13 +327,21 @@ fused_kernel(const ApplyParams P) {
         copy_rows(P, rowidx, rows, (int32_t)crank, (int32_t)csize);
         return;
     }
+    // the tile record and the tile's row ids are fetched side by side (no dependent load)
+    if (P.meta) {
+        if (tid < P.tile_m) rowidx[tid] = P.meta[L.tile_perm + (int64_t)unit * P.tile_m + tid];
+    } else if (tid == 0) {
+        rowidx[0] = unit;
+    }
+    // the tile count sits in one word that every block reads (L2-hot): unused units leave on it
+    const int32_t n_tile = P.meta ? __ldg(P.meta + H_NTILE) : P.T;
     const Tile tl = resolve_unit(P, L, unit);
+    if (unit >= n_tile) return;
     if (!tl.valid) {
         if (!P.meta && unit < P.T) {   // per-token mode: this token has no adapter
             if (crank == 0 && tid == 0 && P.slot_idx[unit] != -1)
                 atomicAdd(&P.pool.status[STATUS_INVALID_TOKENS], 1);
             if (!P.in_place) {
-                if (tid == 0) rowidx[0] = unit;
                 __syncthreads();
                 copy_rows(P, rowidx, 1, (int32_t)crank, (int32_t)csize);
             }
@@ -335,45 +349,38 @@ fused_kernel(const ApplyParams P) {
         return;
     }
     if (tid == 0) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) mbar_init(&bars[i], 1);
+        mbar_init(&bars[BAR_A], 1);
+        mbar_init(&bars[BAR_B], 1);
+        mbar_init(&bars[BAR_X], 1);
         fence_mbar_init();
     }
-    for (int i = tid; i < tl.rows; i += AP_THREADS)
-        rowidx[i] = P.meta ? P.meta[L.perm + tl.row0 + i] : tl.row0 + i;
     __syncthreads();
-    switch (rank_bucket(tl.rank)) {
-        case 8: fused_body<8, 2, 64>(P, tl, smem, crank, csize); break;
-        case 16: fused_body<16, 4, 64>(P, tl, smem, crank, csize); break;
-        case 32: fused_body<32, 4, 64>(P, tl, smem, crank, csize); break;
-        default: fused_body<64, 8, 32>(P, tl, smem, crank, csize); break;
-    }
+    const int32_t b = rank_bucket(tl.rank);
+    if (b <= 16) fused_body<16, 512, 512>(P, tl, smem, crank, csize);
+    else if (b == 32) fused_body<32, 256, 256>(P, tl, smem, crank, csize);
+    else fused_body<64, 256, 256>(P, tl, smem, crank, csize);
 }
 
-// shared memory the kernel needs for pools whose largest rank bucket is RS
+// shared memory for the two weight stages, for pools whose largest rank bucket is RS
 static int32_t stage_bytes_for(int32_t RS) {
-    // per bucket: A + X + B + YB stages (see fused_body)
-    const int32_t b8 = 8 * 512 * 2 + 16 * 512 * 2 + 8 * 512 * 2 + 16 * 512 * 2;
-    const int32_t b16 = 16 * 512 * 2 + 16 * 512 * 2 + 16 * 512 * 2 + 16 * 512 * 2;
-    const int32_t b32 = 32 * 256 * 2 + 16 * 256 * 2 + 32 * 512 * 2 + 16 * 512 * 2;
-    const int32_t b64 = 64 * 256 * 2 + 16 * 256 * 2 + 64 * 256 * 2 + 16 * 256 * 2;
-    int32_t m = b8;
-    if (RS >= 16 && b16 > m) m = b16;
-    if (RS >= 32 && b32 > m) m = b32;
-    if (RS >= 64 && b64 > m) m = b64;
-    return m;
+    const int32_t b16 = 2 * 16 * 512 * 2, b32 = 2 * 32 * 256 * 2, b64 = 2 * 64 * 256 * 2;
+    return RS <= 16 ? b16 : RS == 32 ? (b16 > b32 ? b16 : b32) : b64;
 }
 
 lora_status_t launch_fused(lora_pool_t *pool, ApplyParams &P, cudaStream_t stream) {
-    const int32_t RS = P.RS;
+    const int32_t RS = P.RS < 16 ? 16 : P.RS;
     int32_t rows_cap = P.meta ? P.tile_m : 1;
     rows_cap = (rows_cap + 15) & ~15;
     P.rows_cap = rows_cap;
-    const int32_t part_floats_per_row = RS == 8 ? 16 : RS == 16 ? 32 : RS;   // WPK * RP, worst bucket
+    // partial v: WPK copies of [rows][RP]; WPK * RP is 32 for the <=16 bucket, RP above
+    const int32_t part_floats_per_row = RS == 16 ? 32 : RS;
     P.off_part = FUSED_HEAD_BYTES;
     P.off_vst = P.off_part + rows_cap * part_floats_per_row * 4;
     P.off_stage = (P.off_vst + RS * rows_cap * 4 + 127) & ~127;
-    const int32_t smem = P.off_stage + stage_bytes_for(RS);
+    P.off_x = P.off_stage + stage_bytes_for(RS);
+    int32_t x_rows = ((P.meta ? P.tile_m : 1) + 7) & ~7;
+    if (x_rows > XROWS) x_rows = XROWS;
+    const int32_t smem = P.off_x + x_rows * 512 * 2;   // x stage: up to XROWS rows of 512 columns
 
     // cluster size: as wide a split as the projection supports, narrower when there are many units
     int32_t C = pool->tuning[1];
@@ -393,7 +400,7 @@ lora_status_t launch_fused(lora_pool_t *pool, ApplyParams &P, cudaStream_t strea
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)((P.units + copy_units) * C), 1, 1);
-    cfg.blockDim = dim3(AP_THREADS, 1, 1);
+    cfg.blockDim = dim3(FT, 1, 1);
     cfg.dynamicSmemBytes = (size_t)smem;
     cfg.stream = stream;
     cudaLaunchAttribute at[1];

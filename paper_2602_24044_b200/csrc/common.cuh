@@ -72,7 +72,7 @@ enum { H_T = 0, H_NACTIVE = 1, H_NINVALID = 2, H_NSEG = 3, H_NTILE = 4, H_TILE_M
 struct MetaLayout {
     int32_t cap_seg, cap_tile;
     int64_t perm, seg_slot, seg_start, seg_rank, seg_flags, tile_seg, tile_row0, tile_rows,
-        tile_flags, tile_desc, words;
+        tile_flags, tile_desc, tile_perm, words;
 };
 
 __host__ __device__ inline MetaLayout meta_layout(int32_t T, int32_t num_slots, int32_t tile_m) {
@@ -91,6 +91,7 @@ __host__ __device__ inline MetaLayout meta_layout(int32_t T, int32_t num_slots, 
     L.tile_flags = o; o += L.cap_tile;
     o = (o + 3) & ~(int64_t)3;            // library-private part, 16-byte aligned records
     L.tile_desc = o;  o += 4 * (int64_t)L.cap_tile;   // {slot, row0, rows | rank << 16, scale bits}
+    L.tile_perm = o;  o += (int64_t)L.cap_tile * tile_m;   // tile k's token ids at k * tile_m
     L.words = o;
     return L;
 }

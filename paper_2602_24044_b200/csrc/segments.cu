@@ -86,7 +86,12 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx, int32
             const int32_t t = base + lane;
             const bool hit = t < T && slot_idx[t] == s;
             const uint32_t m = __ballot_sync(0xffffffffu, hit);
-            if (hit) perm[p0 + run + __popc(m & ((1u << lane) - 1u))] = t;
+            if (hit) {
+                const int32_t j = run + __popc(m & ((1u << lane) - 1u));
+                perm[p0 + j] = t;
+                // private copy laid out by tile: tile k of the batch starts at k * tile_m
+                meta[L.tile_perm + (int64_t)tile0[s] * tile_m + j] = t;
+            }
             run += __popc(m);
         }
         __syncwarp();

@@ -82,6 +82,8 @@ def test_segments_bytes_matches_documented_layout():
     words = 16 + T + 4 * cap_seg + 1 + 4 * cap_tile
     public_words = words
     words = (words + 3) // 4 * 4 + 4 * cap_tile          # library-private tile records
+    desc_end = words
+    words += cap_tile * tile_m                           # library-private per-tile row ids
     assert lb.segments_bytes(T, N, tile_m) == 4 * words
     assert lb.segments_bytes(0, N, tile_m) == 4 * 20
     with pytest.raises(lb.LoraError):
@@ -90,7 +92,7 @@ def test_segments_bytes_matches_documented_layout():
     parts = lb.unpack_segments(meta, T, N, tile_m)
     assert parts["perm"][0] == 16 and len(parts["tile_flags"]) == cap_tile
     assert parts["tile_flags"][-1] == public_words - 1
-    assert parts["tile_desc"][-1, -1] == words - 1
+    assert parts["tile_desc"][-1, -1] == desc_end - 1
 
 
 def test_null_handles_are_rejected():
