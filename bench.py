@@ -51,6 +51,8 @@ def parse_args():
                     help="apply path: 0 fused cluster kernel (default), 1 two-phase kernels")
     ap.add_argument("--cluster", type=int, default=None, help="fused path: cluster size 1/2/4/8")
     ap.add_argument("--tile-m", type=int, default=None, help="rows per tile of the segment metadata")
+    ap.add_argument("--tune", nargs="*", default=[], metavar="KEY=VALUE",
+                    help="lora_pool_set_tuning pairs, e.g. 2=1 (no programmatic dependent launch)")
     return ap.parse_args()
 
 
@@ -227,6 +229,9 @@ def main():
         tuning[0] = args.algo
     if args.cluster is not None:
         tuning[1] = args.cluster
+    for kv in args.tune:
+        k, v = kv.split("=")
+        tuning[int(k)] = int(v)
     s = Session(wl, device="cuda:%d" % local, a_layout=lb.A_RANK_MAJOR, tuning=tuning)
     dev = s.device
     xs, ybs, ys, metas = [], [], [], []

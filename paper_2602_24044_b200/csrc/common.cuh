@@ -123,6 +123,7 @@ struct lora_pool {
     std::vector<cudaEvent_t> ready;     // per slot, created on first load
     cudaEvent_t fence = nullptr;        // compute -> load ordering
     int32_t sm_count = 148;
+    uint32_t bucket_mask = 0;           // rank buckets (8/16/32/64 -> bits 0..3) ever loaded into a slot
     int32_t tuning[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 
     // Shapes of the metadata tables built through this handle (the table itself lives on the

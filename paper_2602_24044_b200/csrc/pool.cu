@@ -236,6 +236,8 @@ lora_status_t lora_pool_load_slot(lora_pool_t *pool, int32_t slot, const lora_ad
     set_slot_kernel<<<1, 32, 0, ls>>>(pool->table_dev, slot, r, ad->scale, 1);
     if ((s = count_launch()) != LORA_OK) return s;
     LORA_CUDA_TRY(cudaEventRecord(pool->ready[slot], ls));
+    const int32_t rb = rank_bucket(r);
+    pool->bucket_mask |= rb == 8 ? 1u : rb == 16 ? 2u : rb == 32 ? 4u : 8u;
     pool->table_host[slot].rank = r;
     pool->table_host[slot].scale = ad->scale;
     pool->table_host[slot].loaded = 1;

@@ -13,31 +13,41 @@ namespace lora {
 constexpr int SEG_THREADS = 256;
 constexpr int SEG_WARPS = SEG_THREADS / 32;
 
-__device__ __forceinline__ bool token_active(const PoolView &pool, int32_t s) {
-    return s >= 0 && s < pool.num_slots && pool.table[s].loaded != 0;
-}
-
 __global__ void __launch_bounds__(SEG_THREADS)
-build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx, int32_t T,
-                      int32_t tile_m, int32_t long_min, int32_t *meta) {
+build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int32_t T,
+                      int32_t tile_m, int32_t long_min, int32_t *meta, int32_t staged) {
     extern __shared__ int32_t sm[];
     const int32_t N = pool.num_slots;
     int32_t *cnt = sm;             // [N] tokens per slot
     int32_t *start = cnt + N;      // [N] first position in perm
     int32_t *segid = start + N;    // [N] segment number
     int32_t *tile0 = segid + N;    // [N] first tile number
+    int32_t *occ = tile0 + N;      // [N] slot occupied (copy of the slot table's flag)
+    int32_t *tok = occ + N;        // [T] copy of the token list (only when `staged`)
     __shared__ int32_t warp_tot[3][SEG_WARPS];
     __shared__ int32_t totals[3];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const MetaLayout L = meta_layout(T, N, tile_m);
+    // programmatic dependent launch: the next kernel of the stream may be scheduled now; this one
+    // waits until everything queued before it is complete (no-ops without the launch attribute)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- 1. histogram of active tokens ------------------------------------------------------
-    for (int32_t s = tid; s < N; s += SEG_THREADS) cnt[s] = 0;
+    // The slot flags and (for batches that fit) the token list are copied to shared memory with
+    // independent loads first, so that the scans below do not pay a global round trip per step.
+    for (int32_t s = tid; s < N; s += SEG_THREADS) {
+        cnt[s] = 0;
+        occ[s] = pool.table[s].loaded;
+    }
+    if (staged)
+        for (int32_t t = tid; t < T; t += SEG_THREADS) tok[t] = slot_idx_g[t];
+    const int32_t *slot_idx = staged ? tok : slot_idx_g;
     __syncthreads();
     for (int32_t t = tid; t < T; t += SEG_THREADS) {
         const int32_t s = slot_idx[t];
-        if (token_active(pool, s)) atomicAdd(&cnt[s], 1);
+        if (s >= 0 && s < N && occ[s]) atomicAdd(&cnt[s], 1);
     }
     __syncthreads();
 
@@ -124,7 +134,7 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx, int32
         for (int32_t base = 0; base < T; base += 32) {
             const int32_t t = base + lane;
             const int32_t s = t < T ? slot_idx[t] : -1;
-            const bool inact = t < T && !token_active(pool, s);
+            const bool inact = t < T && !(s >= 0 && s < N && occ[s]);
             const uint32_t m = __ballot_sync(0xffffffffu, inact);
             const uint32_t bad = __ballot_sync(0xffffffffu, inact && s != -1);
             if (inact) perm[n_active + run + __popc(m & ((1u << lane) - 1u))] = t;
@@ -171,14 +181,25 @@ lora_status_t launch_build_segments(lora_pool_t *pool, const int32_t *slot_idx_d
     int grid = (N + SEG_WARPS - 1) / SEG_WARPS;
     if (grid > 2 * pool->sm_count) grid = 2 * pool->sm_count;
     if (grid < 1) grid = 1;
-    const size_t smem = sizeof(int32_t) * 4 * (size_t)N;
+    const int32_t staged = T <= 8192 ? 1 : 0;   // the token list fits beside the per-slot arrays
+    const size_t smem = sizeof(int32_t) * (5 * (size_t)N + (staged ? (size_t)T : 0));
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(build_segments_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return cuda_fail(e);
     }
-    build_segments_kernel<<<grid, SEG_THREADS, smem, stream>>>(pool->view(), slot_idx_dev, T,
-                                                               tile_m, long_min, (int32_t *)meta_dev);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(SEG_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pool->tuning[2] == 1 ? 1 : 0;   // tuning key 2 = 1: programmatic dependent launch
+    LORA_CUDA_TRY(cudaLaunchKernelEx(&cfg, build_segments_kernel, pool->view(), slot_idx_dev, T,
+                                     tile_m, long_min, (int32_t *)meta_dev, staged));
     return count_launch();
 }
 

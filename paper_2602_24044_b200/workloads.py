@@ -192,12 +192,13 @@ def make_config(config: int, rep: int = 0, layers: int = 32) -> Workload:
         N, T = 8, 16
         return Workload("decode_tiny", 0, seed, "bgmv", [(1024, 1024)], N, 8,
                         np.full(N, 8, np.int32), np.full(N, 2.0, np.float32),
-                        np.ones(N, np.int32), rng.integers(0, N, T).astype(np.int32), [0])
+                        np.ones(N, np.int32), rng.integers(0, N, T).astype(np.int32), [0],
+                        tile_m=8)
     if config == 1:
         N, T = 128, 256
         return Workload("decode_q_proj", 1, seed, "bgmv", [(4096, 4096)], N, 16,
                         np.full(N, 16, np.int32), np.full(N, 2.0, np.float32),
-                        np.ones(N, np.int32), bounded_zipf(rng, N, 1.1, T), [0])
+                        np.ones(N, np.int32), bounded_zipf(rng, N, 1.1, T), [0], tile_m=8)
     if config == 2:
         N, R = 64, 32
         lens = lognormal_lengths(rng, R, 512.0, 1.0, 32, 2048)
@@ -227,7 +228,7 @@ def make_config(config: int, rep: int = 0, layers: int = 32) -> Workload:
         return Workload("llama3_8b_step", 4, seed, "bgmv", targets, N, 16,
                         np.full(N, 16, np.int32), np.full(N, 2.0, np.float32),
                         np.ones(N, np.int32), slot_idx, list(range(len(targets))),
-                        swap_victims=victims, info={"layers": layers})
+                        tile_m=8, swap_victims=victims, info={"layers": layers})
     raise ValueError(f"unknown config {config}")
 
 
