@@ -42,7 +42,9 @@ PAPER_CONTEXT = {
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=48000)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3, 4],
+                    help="workload: 1 (default) is the headline decode batch; the others are the parity configurations")
     ap.add_argument("--warmup", type=int, default=160)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=200)
@@ -180,7 +182,7 @@ def run_reference(args):
     from oracle import lora_oracle as orc
     orc.build()
     # each step = one whole batch of the workload through the oracle; at most ~2 minutes in all
-    t = time_oracle(wl, budget_s=120.0, max_reps=max(1, args.steps), warm=max(1, min(args.warmup, 20)))
+    t = time_oracle(wl, budget_s=120.0, max_reps=max(1, args.steps or 48000), warm=max(1, min(args.warmup, 20)))
     line = {"impl": "reference", "metric": METRIC, "value": t["value"], "unit": UNIT,
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "steps_timed": t["reps"], "ms_per_step": t["ms_per_step"], "higher_is_better": True, "scaling": "weak",
@@ -192,6 +194,35 @@ def run_reference(args):
                     "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
+
+
+WORKLOAD_TEXT = {
+    0: "config0 decode BGMV tiny: 16 tokens, 1024->1024, 8 adapters rank 8, uniform slots",
+    1: "config1 decode BGMV: 256 tokens, 4096->4096, 128 resident adapters rank 16, Zipf(1.1) over slots",
+    2: "config2 prefill SGMV: 32 requests, lognormal prompt lengths (median 512, clip 32..2048), "
+       "4096->14336 and 14336->4096, 64 adapters ranks {8,16,32}",
+    3: "config3 mixed chunked prefill SGMV: 512 decode tokens + 4 chunks of 512, fused QKV 4096->6144, "
+       "384 adapters ranks {8,16,32,64}, Zipf(0.9)",
+    4: "config4 full 32-layer decode step, Llama-3-8B shapes, LoRA on all 7 projections, 256 tokens, "
+       "256 adapters rank 16, Zipf(1.1)",
+}
+
+
+def case_workload(cfg):
+    """The workload object of a configuration, with the rotation of independent copies that keeps
+    every step cold in L2 for the small ones."""
+    from paper_2602_24044_b200 import workloads as W
+    wl = W.make_config(cfg)
+    rotation = 1
+    if cfg in (0, 1):
+        rotation = ROTATION
+    elif cfg == 3:
+        rotation = 2
+    n_proj = len(wl.targets)
+    if rotation > 1:
+        wl.targets = wl.targets * rotation
+        wl.calls = list(range(len(wl.targets)))
+    return wl, rotation, n_proj
 
 
 def main():
@@ -219,10 +250,10 @@ def main():
     if world > 1:
         dist.barrier()
 
-    wl = bench_workload()
+    cfg = args.config
+    wl, rotation, n_proj = case_workload(cfg)
     if args.tile_m is not None:
         wl.tile_m = args.tile_m
-    d_in, d_out = wl.targets[0]
     T = wl.T
     tuning = {}
     if args.algo is not None:
@@ -232,40 +263,67 @@ def main():
     for kv in args.tune:
         k, v = kv.split("=")
         tuning[int(k)] = int(v)
-    s = Session(wl, device="cuda:%d" % local, a_layout=lb.A_RANK_MAJOR, tuning=tuning)
-    dev = s.device
-    xs, ybs, ys, metas = [], [], [], []
+    dev = torch.device("cuda", local)
+    if cfg == 4:
+        # 256 slots x 83.9 MB: every slot is filled by a swap-in from ONE pinned host adapter (the
+        # values do not influence the timing; addresses and sizes are those of 256 distinct adapters)
+        s = Session(wl, device="cuda:%d" % local, slots=[], tuning=tuning)
+        blobs = s.host_adapter(0, lb.A_RANK_MAJOR)
+        for slot in range(wl.num_slots):
+            s.load_slot(slot, a_layout=lb.A_RANK_MAJOR, src_slot=0, blobs=blobs)
+        torch.cuda.synchronize()
+    else:
+        s = Session(wl, device="cuda:%d" % local, a_layout=lb.A_RANK_MAJOR, tuning=tuning)
+
+    # device buffers: one set per rotation index; a set holds the step's applies in order
+    act_sets = min(rotation, ROTATION) if cfg != 4 else 4     # config 4: activations of 4 layers cycle
+    sets, metas = [], []
     meta_words = lb.segments_bytes(T, wl.num_slots, wl.tile_m) // 4
-    for c in range(ROTATION):
-        x_h, yb_h = wl.activations(c)
-        xs.append(bf16_tensor(x_h, dev))
-        ybs.append(bf16_tensor(yb_h, dev))
-        ys.append(torch.empty((T, d_out), dtype=torch.bfloat16, device=dev))
+    n_sets = rotation if cfg != 4 else 1
+    acts = {}
+    for r in range(n_sets):
+        calls = []
+        for j in range(len(wl.calls) // n_sets):
+            call = r * (len(wl.calls) // n_sets) + j
+            key = call if cfg != 4 else call % (7 * act_sets)
+            if key not in acts:
+                x_h, yb_h = wl.activations(key)
+                acts[key] = (bf16_tensor(x_h, dev), bf16_tensor(yb_h, dev),
+                             torch.empty(yb_h.shape, dtype=torch.bfloat16, device=dev))
+            x, yb, y = acts[key]
+            calls.append((s.target_pos[wl.calls[call]], x, yb, y))
+        sets.append(calls)
         metas.append(torch.empty(meta_words, dtype=torch.int32, device=dev))
     torch.cuda.synchronize()
+    sgmv = wl.kind == "sgmv"
+
+    def apply_calls(r):
+        for tp, x, yb, y in sets[r]:
+            if sgmv:
+                lb.sgmv_apply(s.pool, tp, x, x.shape[1], yb, yb.shape[1], y, y.shape[1], metas[r], T, s.ws,
+                              stream=s.compute)
+            else:
+                lb.bgmv_apply(s.pool, tp, x, x.shape[1], yb, yb.shape[1], y, y.shape[1], s.slot_idx_dev,
+                              T, metas[r], s.ws, stream=s.compute)
 
     def step(i):
-        c = i % ROTATION
-        lb.build_segments(s.pool, s.slot_idx_dev, T, wl.tile_m, wl.long_min, metas[c],
-                          stream=s.compute)
-        lb.bgmv_apply(s.pool, c, xs[c], d_in, ybs[c], d_out, ys[c], d_out, s.slot_idx_dev, T,
-                      metas[c], s.ws, stream=s.compute)
+        r = i % n_sets
+        lb.build_segments(s.pool, s.slot_idx_dev, T, wl.tile_m, wl.long_min, metas[r], stream=s.compute)
+        apply_calls(r)
 
     def apply_only(i):
-        c = i % ROTATION
-        lb.bgmv_apply(s.pool, c, xs[c], d_in, ybs[c], d_out, ys[c], d_out, s.slot_idx_dev, T,
-                      metas[c], s.ws, stream=s.compute)
+        apply_calls(i % n_sets)
 
     def capture(fn):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=s.compute):
-            for i in range(ROTATION):
+            for i in range(n_sets):
                 fn(i)
         return g
 
     # warm-up (also sets kernel attributes before capture)
     with torch.cuda.stream(s.compute):
-        for i in range(max(args.warmup, 3)):
+        for i in range(max(min(args.warmup, 8 * n_sets), 3)):
             step(i)
     torch.cuda.synchronize()
     l0 = lb.launch_count()
@@ -276,19 +334,20 @@ def main():
 
     def run_steps(K, graph, fn):
         with torch.cuda.stream(s.compute):
-            for _ in range(K // ROTATION):
+            for _ in range(K // n_sets):
                 graph.replay()
-            for i in range(K % ROTATION):
+            for i in range(K % n_sets):
                 fn(i)
 
-    run_steps(ROTATION * 4, g_step, step)
+    K = args.steps if args.steps is not None else {0: 48000, 1: 48000, 2: 300, 3: 3000, 4: 100}[cfg]
+    W_ = max(args.warmup, 3)
+    run_steps(min(W_, max(3, K // 4)), g_step, step)
     torch.cuda.synchronize()
 
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    K = args.steps
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if world > 1:
         dist.barrier()
@@ -298,7 +357,7 @@ def main():
     run_steps(K, g_step, step)
     e1.record(s.compute)
     torch.cuda.synchronize()
-    launches = (K // ROTATION) * launches_per_rotation + (lb.launch_count() - l0)
+    launches = (K // n_sets) * launches_per_rotation + (lb.launch_count() - l0)
     if world > 1:
         dist.barrier()
     ms = e0.elapsed_time(e1)
@@ -307,33 +366,63 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
 
-    # the apply alone (dominant kernels), same rotation, for the roofline figure
-    Kr = max(ROTATION, min(K, 16000) // ROTATION * ROTATION)
+    # the applies alone (dominant kernel), same rotation, for the roofline figure
+    Kr = max(n_sets, min(K, 16000) // n_sets * n_sets)
     r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     r0.record(s.compute)
     run_steps(Kr, g_apply, apply_only)
     r1.record(s.compute)
     torch.cuda.synchronize()
-    apply_ms = r0.elapsed_time(r1) / Kr
+    calls_per_step = len(sets[0])
+    apply_ms = r0.elapsed_time(r1) / Kr / calls_per_step
     clocks = sampler.stop() if rank == 0 else None
 
+    # swap-in on the side stream while steps run (config 4: 16 misses per step)
+    swap = None
+    if cfg == 4 and rank == 0:
+        blobs = s.host_adapter(0, lb.A_RANK_MAJOR)
+        adapter_bytes = sum(int(t.numel()) * 2 for t in blobs[0] + blobs[1])
+        steps_sw = 5
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0e, l1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        ev0.record(s.compute)
+        l0e.record(s.load)
+        for i in range(steps_sw):
+            for v in wl.swap_victims:
+                lb.pool_load_slot(s.pool, v, int(wl.ranks[v]), float(wl.scales[v]), blobs[0], blobs[1],
+                                  lb.A_RANK_MAJOR, s.load, None, True)
+            run_steps(1, g_step, step)
+        ev1.record(s.compute)
+        l1e.record(s.load)
+        torch.cuda.synchronize()
+        swap = {"misses_per_step": len(wl.swap_victims), "adapter_bytes": adapter_bytes,
+                "h2d_GBps": steps_sw * len(wl.swap_victims) * adapter_bytes / (l0e.elapsed_time(l1e) * 1e6),
+                "ms_per_step_compute_while_loading": ev0.elapsed_time(ev1) / steps_sw,
+                "ms_per_step_of_loads": l0e.elapsed_time(l1e) / steps_sw,
+                "note": "victim slots are not referenced by the step's tokens; loads run on the side "
+                        "stream concurrently with the compute stream"}
+
     # end to end: host buffers in, host result out, every step (C entry point lora_apply_host)
-    xh = [bf16_tensor(wl.activations(c)[0], pin=True) for c in range(2)]
-    ybh = [bf16_tensor(wl.activations(c)[1], pin=True) for c in range(2)]
-    yh = [torch.empty((T, d_out), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+    d_in0, d_out0 = wl.targets[wl.calls[0]]
+    Ke = args.e2e_steps if cfg in (0, 1) else max(3, min(args.e2e_steps, 10))
+    x_h, yb_h = wl.activations(0)
+    xh = [bf16_tensor(x_h, pin=True) for _ in range(2)]
+    ybh = [bf16_tensor(yb_h, pin=True) for _ in range(2)]
+    yh = [torch.empty((T, d_out0), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
     sh = torch.from_numpy(wl.slot_idx.copy()).pin_memory()
     sd = torch.empty(T, dtype=torch.int32, device=dev)
+    tp0, xd, ybd, yd = sets[0][0]
 
     def e2e_step(i):
         c = i % 2
-        lb.apply_host(s.pool, i % ROTATION, 0, xh[c], ybh[c], yh[c], sh, T, wl.tile_m, wl.long_min,
-                      xs[c], ybs[c], ys[c], sd, metas[c], s.ws, s.compute)
+        lb.apply_host(s.pool, tp0, 1 if sgmv else 0, xh[c], ybh[c], yh[c], sh, T, wl.tile_m, wl.long_min,
+                      xd, ybd, yd, sd, metas[0], s.ws, s.compute)
 
-    for i in range(5):
+    for i in range(3):
         e2e_step(i)
     torch.cuda.synchronize()
-    Ke = args.e2e_steps
     if world > 1:
         dist.barrier()
     t0 = time.perf_counter()
@@ -345,8 +434,8 @@ def main():
         t = torch.tensor([e2e_s], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_s = float(t.item())
-    h2d = 2 * T * (d_in + d_out) + 4 * T
-    d2h = 2 * T * d_out
+    h2d = 2 * T * (d_in0 + d_out0) + 4 * T
+    d2h = 2 * T * d_out0
 
     if rank != 0:
         s.close()
@@ -355,38 +444,46 @@ def main():
         return
 
     peak, peak_kind = measured_peak()
-    alg = algorithmic_bytes(wl)
-    achieved = alg / (apply_ms * 1e-3) / 1e9
+    alg_calls = [algorithmic_bytes(wl, wl.calls[j]) for j in range(calls_per_step)]
+    alg = sum(alg_calls)
+    achieved = alg / calls_per_step / (apply_ms * 1e-3) / 1e9
+    fused = tuning.get(0) != 1
     line = {
         "metric": METRIC, "value": world * T * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": K, "warmup": args.warmup, "ms_per_step": ms / K, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in/out, fp32 accumulate",
         "data": "synthetic",
         "config": {
-            "workload": "config1 decode BGMV: 256 tokens, 4096->4096, 128 resident adapters rank 16, "
-                        "Zipf(1.1) over slots (%d distinct)" % len(wl.distinct_slots()),
-            "step": "lora_build_segments + lora_bgmv_apply (grouped), one layer step",
-            "cache": "cold: %d rotating input/weight sets (%.0f MB touched per rotation, L2 is 126 MB)"
-                     % (ROTATION, ROTATION * alg / 1e6),
-            "launch": "CUDA graph of %d consecutive steps replayed" % ROTATION,
+            "workload": WORKLOAD_TEXT[cfg] + " (%d tokens, %d distinct adapters)" % (T, len(wl.distinct_slots())),
+            "step": "lora_build_segments + %d x %s, one %s" % (
+                calls_per_step, "lora_sgmv_apply" if sgmv else "lora_bgmv_apply (grouped)",
+                "layer step" if cfg != 4 else "32-layer step (tokens/s per layer step = value x 32)"),
+            "cache": ("cold: %d rotating input/weight sets (%.0f MB touched per rotation, L2 is 126 MB)"
+                      % (n_sets, n_sets * alg / 1e6)) if n_sets > 1 else
+                     "cold: one step touches %.0f MB, more than the 126 MB L2" % (alg / 1e6),
+            "launch": "CUDA graph of %d consecutive step(s) replayed" % n_sets,
             "multi_gpu": "independent replicas, no collective",
         },
         "roofline": {
             "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
             "frac": achieved / peak, "peak_source": "%s copy bandwidth" % peak_kind,
             "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-            "kernel": ("lora_bgmv_apply: shrink_kernel + expand_kernel (two launches)"
-                       if tuning.get(0) == 1 else "lora_bgmv_apply: fused_kernel (one launch)"),
-            "algorithmic_bytes_per_launch": alg,
+            "kernel": ("fused_kernel (one launch per apply and rank bucket)" if fused
+                       else "shrink_kernel + expand_kernel (two launches per apply)"),
+            "algorithmic_bytes_per_launch": alg / calls_per_step,
             "us_per_launch": apply_ms * 1e3, "traffic": None,
+            "averaged_over": "%d applies per step" % calls_per_step,
         },
         "step_GBps": alg / (ms / K * 1e-3) / 1e9,
         "e2e": {"value": world * T * Ke / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "api": "lora_apply_host", "steps": Ke},
+                "d2h_bytes_per_step": d2h, "api": "lora_apply_host (first projection of the step)",
+                "steps": Ke},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "paper_context": PAPER_CONTEXT,
     }
+    if swap is not None:
+        line["swap_in"] = swap
     if not args.no_cpu_baseline:
         line["cpu_baseline"] = {k: v for k, v in time_oracle(wl).items()
                                 if k not in ("ms_per_step", "reps")}
