@@ -59,13 +59,21 @@ static lora_status_t apply_common(lora_pool_t *pool, int32_t target, const void 
                                   const void *yb, int64_t ldyb, void *y, int64_t ldy,
                                   const int32_t *slot_idx_dev, int32_t T, const void *meta,
                                   int32_t tile_m, void *workspace, size_t workspace_bytes,
-                                  cudaStream_t stream) {
+                                  cudaStream_t stream, bool use_tc) {
     ApplyParams P;
     fill_apply_params(pool, P, target, x, ldx, yb, ldyb, y, ldy, slot_idx_dev, T, meta, tile_m);
     // the workspace contract holds on every path, whether or not the chosen kernels use it
     if (!workspace || workspace_bytes < (size_t)T * P.RS * sizeof(float))
         return LORA_ERR_BUFFER_TOO_SMALL;
     if (pool->tuning[0] == 1) return launch_twophase(pool, P, workspace, workspace_bytes, stream);
+    // prefill batches: full tiles of 128 consecutive tokens go to the tensor-core kernels
+    // (tuning key 4 = 1 keeps everything on the fused kernel)
+    if (use_tc && pool->tuning[4] != 1) {
+        bool handled = false;
+        lora_status_t s = launch_tc_long_tiles(pool, P, workspace, workspace_bytes, stream, &handled);
+        if (s != LORA_OK) return s;
+        P.path_filter = handled ? 1 : 0;
+    }
     return launch_fused(pool, P, stream);
 }
 }  // namespace lora
@@ -95,7 +103,7 @@ lora_status_t lora_bgmv_apply(lora_pool_t *pool, int32_t target, const void *x, 
     DeviceGuard guard(pool->device);
     if (!guard.ok) return cuda_fail(cudaErrorInvalidDevice);
     return apply_common(pool, target, x, ldx, y_base, ldyb, y, ldy, slot_idx_dev, T, meta, tile_m,
-                        workspace, workspace_bytes, (cudaStream_t)stream);
+                        workspace, workspace_bytes, (cudaStream_t)stream, false);
 }
 
 lora_status_t lora_sgmv_apply(lora_pool_t *pool, int32_t target, const void *x, int64_t ldx,
@@ -110,7 +118,7 @@ lora_status_t lora_sgmv_apply(lora_pool_t *pool, int32_t target, const void *x, 
     DeviceGuard guard(pool->device);
     if (!guard.ok) return cuda_fail(cudaErrorInvalidDevice);
     return apply_common(pool, target, x, ldx, y_base, ldyb, y, ldy, nullptr, T, meta, tile_m,
-                        workspace, workspace_bytes, (cudaStream_t)stream);
+                        workspace, workspace_bytes, (cudaStream_t)stream, true);
 }
 
 lora_status_t lora_apply_host(lora_pool_t *pool, int32_t target, int32_t kind, const void *x_host,

@@ -96,7 +96,7 @@ __device__ __forceinline__ Tile resolve_unit(const ApplyParams &P, const MetaLay
         if (d.x < 0) return t;   // unused entry
         t.slot = d.x;
         t.row0 = d.y;
-        t.rows = d.z & 0xffff;
+        t.rows = d.z & 0x7fff;
         t.rank = d.z >> 16;
         t.scale = __int_as_float(d.w);
         t.valid = true;
@@ -139,6 +139,8 @@ static inline int32_t next_pow2(int32_t v) {
 lora_status_t launch_twophase(lora_pool_t *pool, ApplyParams &P, void *workspace,
                               size_t workspace_bytes, cudaStream_t stream);
 lora_status_t launch_fused(lora_pool_t *pool, ApplyParams &P, cudaStream_t stream);
+lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, void *workspace,
+                                   size_t workspace_bytes, cudaStream_t stream, bool *handled);
 lora_status_t launch_build_segments(lora_pool_t *pool, const int32_t *slot_idx_dev, int32_t T,
                                     int32_t tile_m, int32_t long_min, void *meta_dev,
                                     cudaStream_t stream);

@@ -436,11 +436,16 @@ fused_kernel(const ApplyParams P) {
             const int4 d = __ldg(reinterpret_cast<const int4 *>(P.meta + P.moff_desc) + unit);
             tl.slot = d.x;
             tl.row0 = d.y;
-            tl.rows = d.z & 0xffff;
+            tl.rows = d.z & 0x7fff;
             tl.rank = d.z >> 16;
             tl.scale = __int_as_float(d.w);
             tl.valid = d.x >= 0;
             if (unit >= n_tile) break;
+            // full tiles of consecutive tokens belong to the tensor-core kernels when those ran
+            if (P.path_filter && tl.rows == 128 && ((d.z >> 15) & 1)) {
+                __syncthreads();
+                continue;
+            }
         } else {
             if (tid == 0) rowidx[0] = unit;
             MetaLayout L;

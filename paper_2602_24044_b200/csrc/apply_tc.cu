@@ -1,0 +1,595 @@
+// Tensor-core path of lora_sgmv_apply for LONG tiles: 128 consecutive tokens of one adapter
+// (prefill / chunked-prefill segments), y = y_base + s_i * (x . A_i) . B_i (paper Section 2.2).
+//
+// Such a tile is a dense contraction, so it runs on the 5th-generation tensor cores:
+//   tc_shrink_kernel  V_part[128, r] = X[128, K-slice] . A_i[r, K-slice]^T
+//       X and A_i tiles arrive by TMA (128-byte swizzle) through a 4-stage mbarrier ring; one
+//       thread issues tcgen05.mma (M = 128, N = rank bucket, K = 16) with the accumulator in
+//       tensor memory; the partial of each K-slice goes to the fp32 workspace.
+//   tc_expand_kernel  Y[128, N-slice] = Y_base + s * V . B_i[r, N-slice]
+//       V = sum of the partials, carried as a high and a low bf16 part (two MMAs, ~16 mantissa
+//       bits); per 64-column block one TMA load of the B_i tile and of the y_base tile, MMA into a
+//       ring of tensor-memory accumulators, epilogue tcgen05.ld -> fused scale + residual add ->
+//       bf16 written in place into the y_base tile -> TMA store.
+// Both kernels are HBM-bound streaming kernels: the tensor cores only keep the arithmetic off the
+// critical path.  Every wait on an mbarrier is bounded; on expiry the block records it in the
+// pool's status word, frees its tensor memory and leaves without storing.
+// All other tiles (short, ragged or scattered) are handled by the fused kernel.
+#include <cuda.h>
+
+#include <cstdio>
+#include <cstdlib>
+
+#include "apply_common.cuh"
+
+namespace lora {
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+namespace tc {
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded wait: gives up after a fixed number of polls instead of spinning for ever
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+    for (uint32_t i = 0; i < (1u << 18); ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1,
+                                            uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, "
+        "%3}], [%4];" ::"r"(smem_u32(dst)),
+        "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int c0, int c1, int c2,
+                                            uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, "
+        "%3, %4}], [%5];" ::"r"(smem_u32(dst)),
+        "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int c0, int c1, const void *src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map),
+                 "r"(c0), "r"(c1), "r"(smem_u32(src))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+// D[tmem] (+)= A[smem desc] . B[smem desc], bf16 x bf16 -> fp32, issued by one thread
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                     uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// the mbarrier receives one arrival when every MMA issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                     smem_u32(bar))
+                 : "memory");
+}
+// 32 lanes x 16 consecutive columns of tensor memory -> 16 registers per thread (lane = thread)
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, "
+        "%14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// shared-memory matrix descriptor (start address, leading / stride byte offsets in 16-byte units,
+// descriptor version 1, layout type in the top three bits)
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes,
+                                              uint32_t layout_type) {
+    uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)layout_type << 61;
+    return d;
+}
+constexpr uint32_t LAYOUT_NONE = 0, LAYOUT_SW128 = 2;
+// instruction descriptor: fp32 accumulator, bf16 A and B, majors, N / 8, M / 16
+__host__ __device__ constexpr uint32_t instr_desc(uint32_t M, uint32_t N, uint32_t a_mn_major,
+                                                  uint32_t b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn_major << 15) | (b_mn_major << 16) | ((N >> 3) << 17) |
+           ((M >> 4) << 24);
+}
+}  // namespace tc
+
+constexpr int TC_THREADS = 128;
+constexpr int TC_ROWS = 128;       // rows of a long tile
+constexpr int SH_STAGES = 4;       // shrink: ring of (x tile, A tile) stages
+constexpr int XT_BYTES = TC_ROWS * 128;   // 128 rows x 64 bf16
+
+struct TcParams {
+    PoolView pool;
+    TargetView tv;
+    const int32_t *meta;
+    float *ws;              // [KS][T][RS] fp32 partial v
+    int32_t T, RS, KS, NS;
+    int32_t moff_perm, moff_desc;
+    int32_t target_rows;    // r_max: rows of a slot's matrices
+};
+
+// tile record -> (valid long tile of this bucket?, slot, first token, position in perm, rank, scale)
+struct LongTile {
+    int32_t slot, t0, row0, rank;
+    float scale;
+    bool ok;
+};
+__device__ __forceinline__ LongTile long_tile(const TcParams &P, int32_t unit, int32_t bucket) {
+    LongTile lt;
+    lt.ok = false;
+    const int32_t n_tile = __ldg(P.meta + H_NTILE);
+    if (unit >= n_tile) return lt;
+    const int4 d = __ldg(reinterpret_cast<const int4 *>(P.meta + P.moff_desc) + unit);
+    const int32_t rows = d.z & 0x7fff, contiguous = (d.z >> 15) & 1, rank = d.z >> 16;
+    if (d.x < 0 || rows != TC_ROWS || !contiguous) return lt;
+    const int32_t b = rank_bucket(rank);
+    if ((b <= 16 ? 16 : b) != bucket) return lt;
+    lt.slot = d.x;
+    lt.row0 = d.y;
+    lt.rank = rank;
+    lt.scale = __int_as_float(d.w);
+    lt.t0 = __ldg(P.meta + P.moff_perm + d.y);
+    lt.ok = true;
+    return lt;
+}
+
+// ---------------------------------------------------------------------------------------------
+// shrink
+// ---------------------------------------------------------------------------------------------
+template <int RP>
+__global__ void __launch_bounds__(TC_THREADS)
+tc_shrink_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_x,
+                 const __grid_constant__ CUtensorMap map_a) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    // the swizzled tiles want 1024-byte aligned bases
+    unsigned char *smem = reinterpret_cast<unsigned char *>(
+        ((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    constexpr int AT_BYTES = RP * 128;               // RP rank rows x 64 bf16
+    constexpr int STAGE = XT_BYTES + ((AT_BYTES + 1023) & ~1023);
+    constexpr uint32_t TMEM_COLS = RP < 32 ? 32 : RP;
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + SH_STAGES * STAGE);
+    uint64_t *empty = full + SH_STAGES;
+    uint64_t *done = empty + SH_STAGES;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(done + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const LongTile lt = long_tile(P, blockIdx.x, RP);
+    if (!lt.ok) return;
+    const int32_t ks = blockIdx.y;
+    // K-blocks of 64 columns owned by this block
+    const int32_t nkb_all = (P.tv.d_in + 63) / 64;
+    const int32_t per = (nkb_all + P.KS - 1) / P.KS;
+    const int32_t kb0 = min(ks * per, nkb_all), kb1 = min(kb0 + per, nkb_all);
+    const int32_t nkb = kb1 - kb0;
+
+    if (tid == 0) {
+        for (int s = 0; s < SH_STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
+        tc::mbar_init(done, 1);
+        tc::fence_mbar_init();
+    }
+    if (warp == 0) {
+        tc::tmem_alloc(tmem_slot, TMEM_COLS);
+        tc::tmem_relinquish();
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    bool ok = true;
+
+    if (tid == 0 && nkb > 0) {
+        constexpr uint32_t IDESC = tc::instr_desc(128, RP, 0, 0);
+        auto issue_load = [&](int32_t i) {
+            const int s = i % SH_STAGES;
+            unsigned char *st = smem + s * STAGE;
+            tc::mbar_expect_tx(&full[s], XT_BYTES + AT_BYTES);
+            tc::tma_load_2d(st, &map_x, (kb0 + i) * 64, lt.t0, &full[s]);
+            tc::tma_load_3d(st + XT_BYTES, &map_a, (kb0 + i) * 64, 0, lt.slot, &full[s]);
+        };
+        for (int32_t i = 0; i < nkb && i < SH_STAGES; ++i) issue_load(i);
+        for (int32_t i = 0; i < nkb && ok; ++i) {
+            const int s = i % SH_STAGES;
+            const uint32_t ph = (uint32_t)(i / SH_STAGES) & 1u;
+            ok = tc::mbar_wait(&full[s], ph);
+            if (!ok) break;
+            tc::tc_fence_after();
+            const uint32_t xa = tc::smem_u32(smem + s * STAGE), aa = xa + XT_BYTES;
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4) {   // four K = 16 steps inside the 128-byte swizzle atom
+                const uint64_t ad = tc::smem_desc(xa + k4 * 32, 16, 1024, tc::LAYOUT_SW128);
+                const uint64_t bd = tc::smem_desc(aa + k4 * 32, 16, 1024, tc::LAYOUT_SW128);
+                tc::umma(tmem, ad, bd, IDESC, (i > 0 || k4 > 0) ? 1u : 0u);
+            }
+            tc::umma_commit(&empty[s]);
+            if (i + SH_STAGES < nkb) {       // refill this stage once the MMAs have read it
+                ok = tc::mbar_wait(&empty[s], ph);
+                if (ok) issue_load(i + SH_STAGES);
+            }
+        }
+        tc::umma_commit(done);
+    }
+    __syncwarp();
+    if (nkb > 0) {
+        if (!tc::mbar_wait(done, 0)) ok = false;
+    }
+    tc::tc_fence_after();
+    // accumulator -> fp32 partial in the workspace (thread = row of the tile)
+    const int32_t m = warp * 32 + lane;
+    float *dst = P.ws + ((int64_t)ks * P.T + lt.row0 + m) * P.RS;
+    const bool all_ok = __syncthreads_and(ok ? 1 : 0) != 0;
+    if (all_ok) {
+#pragma unroll
+        for (int c = 0; c < RP; c += 16) {
+            uint32_t r[16];
+            if (nkb > 0) {
+                tc::tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + c, r);
+                tc::tmem_ld_wait();
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) r[i] = 0u;
+            }
+#pragma unroll
+            for (int i = 0; i < 16; i += 4)
+                *reinterpret_cast<uint4 *>(dst + c + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+        }
+    } else if (tid == 0) {
+        atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tc::tmem_dealloc(tmem, TMEM_COLS);
+}
+
+// ---------------------------------------------------------------------------------------------
+// expand
+// ---------------------------------------------------------------------------------------------
+template <int RP>
+struct ExpandCfg {
+    static constexpr int STAGES = RP == 64 ? 4 : 6;
+    static constexpr int BT_BYTES = RP * 128;                       // RP rank rows x 64 columns
+    static constexpr int STAGE = XT_BYTES + ((BT_BYTES + 1023) & ~1023);   // y_base/out tile + B tile
+    static constexpr int V_BYTES = TC_ROWS * RP * 2;                // one bf16 copy of v
+    static constexpr int SMEM = 2 * V_BYTES + STAGES * STAGE + 256 + 1024;
+    static constexpr uint32_t TMEM_COLS = STAGES == 4 ? 256 : 512;  // ring of 64-column accumulators
+};
+
+template <int RP>
+__global__ void __launch_bounds__(TC_THREADS)
+tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
+                 const __grid_constant__ CUtensorMap map_yb, const __grid_constant__ CUtensorMap map_y) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    using C = ExpandCfg<RP>;
+    constexpr int S = C::STAGES;
+    // the swizzled tiles want 1024-byte aligned bases
+    unsigned char *smem = reinterpret_cast<unsigned char *>(
+        ((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char *stages = smem;                                   // [S][y_base tile | B tile]
+    unsigned char *Vh = smem + S * C::STAGE;                        // core-matrix layout, see below
+    unsigned char *Vl = Vh + C::V_BYTES;
+    uint64_t *full = reinterpret_cast<uint64_t *>(Vl + C::V_BYTES);
+    uint64_t *mma_done = full + S;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(mma_done + S);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const LongTile lt = long_tile(P, blockIdx.x, RP);
+    if (!lt.ok) return;
+    // 64-column blocks of d_out owned by this block
+    const int32_t nblk_all = (P.tv.d_out + 63) / 64;
+    const int32_t per = (nblk_all + P.NS - 1) / P.NS;
+    const int32_t b0 = min((int32_t)blockIdx.y * per, nblk_all), b1 = min(b0 + per, nblk_all);
+    const int32_t nblk = b1 - b0;
+    if (nblk <= 0) return;
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&mma_done[s], 1); }
+        tc::fence_mbar_init();
+    }
+    if (warp == 0) {
+        tc::tmem_alloc(tmem_slot, C::TMEM_COLS);
+        tc::tmem_relinquish();
+    }
+    // v = sum of the K-slice partials (in order); thread = row.  Stored as bf16 high and low parts
+    // in the no-swizzle K-major layout: 8 x 8 core matrices of 128 bytes, the core matrix of row
+    // group mg and rank group kg at (kg * 16 + mg) * 128 bytes.
+    {
+        const int32_t m = tid;
+        const float *src = P.ws + ((int64_t)lt.row0 + m) * P.RS;
+        const int64_t ks_stride = (int64_t)P.T * P.RS;
+#pragma unroll
+        for (int kg = 0; kg < RP / 8; ++kg) {
+            float v[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[e] = 0.0f;
+            for (int32_t q = 0; q < P.KS; ++q) {
+                const float4 a = *reinterpret_cast<const float4 *>(src + q * ks_stride + kg * 8);
+                const float4 b = *reinterpret_cast<const float4 *>(src + q * ks_stride + kg * 8 + 4);
+                v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
+                v[4] += b.x; v[5] += b.y; v[6] += b.z; v[7] += b.w;
+            }
+            uint32_t hi[4], lo[4];
+#pragma unroll
+            for (int e = 0; e < 8; e += 2) {
+                const float v0 = kg * 8 + e < lt.rank ? v[e] : 0.0f;
+                const float v1 = kg * 8 + e + 1 < lt.rank ? v[e + 1] : 0.0f;
+                const __nv_bfloat16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
+                hi[e / 2] = pack2(__bfloat162float(h0), __bfloat162float(h1));
+                lo[e / 2] = pack2(v0 - __bfloat162float(h0), v1 - __bfloat162float(h1));
+            }
+            const int off = (kg * 16 + (m >> 3)) * 128 + (m & 7) * 16;
+            *reinterpret_cast<uint4 *>(Vh + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4 *>(Vl + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+    }
+    tc::fence_proxy_async();     // v was written with ordinary stores and is read by the MMA unit
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    bool ok = true;
+
+    constexpr uint32_t IDESC = tc::instr_desc(128, 64, 0, 1);   // A = v (K-major), B = B_i tile (N-major)
+    auto issue_load = [&](int32_t j) {
+        const int s = j % S;
+        unsigned char *st = stages + s * C::STAGE;
+        tc::mbar_expect_tx(&full[s], XT_BYTES + C::BT_BYTES);
+        tc::tma_load_2d(st, &map_yb, (b0 + j) * 64, lt.t0, &full[s]);
+        tc::tma_load_3d(st + XT_BYTES, &map_b, (b0 + j) * 64, 0, lt.slot, &full[s]);
+    };
+    auto issue_mma = [&](int32_t j) -> bool {
+        const int s = j % S;
+        if (!tc::mbar_wait(&full[s], (uint32_t)(j / S) & 1u)) return false;
+        tc::tc_fence_after();
+        const uint32_t ba = tc::smem_u32(stages + s * C::STAGE + XT_BYTES);
+        const uint32_t vh = tc::smem_u32(Vh), vl = tc::smem_u32(Vl);
+        const int32_t ksteps = (lt.rank + 15) >> 4;
+        for (int32_t k = 0; k < ksteps; ++k) {
+            // v: two rank groups per step, 2048 bytes apart; B tile: 16 rank rows = 2048 bytes per step
+            const uint64_t bd = tc::smem_desc(ba + k * 2048, 16, 1024, tc::LAYOUT_SW128);
+            tc::umma(tmem + s * 64, tc::smem_desc(vh + k * 4096, 2048, 128, tc::LAYOUT_NONE), bd, IDESC,
+                     k > 0 ? 1u : 0u);
+            tc::umma(tmem + s * 64, tc::smem_desc(vl + k * 4096, 2048, 128, tc::LAYOUT_NONE), bd, IDESC, 1u);
+        }
+        tc::umma_commit(&mma_done[s]);
+        return true;
+    };
+
+    if (tid == 0) {
+        for (int32_t j = 0; j < nblk && j < S - 1; ++j) issue_load(j);
+        ok = issue_mma(0);
+    }
+    for (int32_t j = 0; j < nblk; ++j) {
+        const int s = j % S;
+        if (tid == 0 && ok && j + 1 < nblk) ok = issue_mma(j + 1);   // next block's MMAs run under this epilogue
+        ok = __syncthreads_and(ok ? 1 : 0) != 0;
+        if (!ok) break;
+        if (!tc::mbar_wait(&mma_done[s], (uint32_t)(j / S) & 1u)) ok = false;
+        tc::tc_fence_after();
+        // epilogue: thread = row; the y_base tile (128-byte swizzle) is updated in place
+        unsigned char *tile = stages + s * C::STAGE;
+        const int m = warp * 32 + lane;
+#pragma unroll
+        for (int c = 0; c < 64; c += 16) {
+            uint32_t r[16];
+            tc::tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + s * 64 + c, r);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int chunk = (c >> 3) + h;
+                uint4 *p = reinterpret_cast<uint4 *>(tile + m * 128 + ((chunk ^ (m & 7)) << 4));
+                float acc[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] = __uint_as_float(r[h * 8 + e]);
+                *p = finish8(acc, *p, lt.scale);
+            }
+        }
+        tc::fence_proxy_async();    // the tile is read by the TMA store
+        tc::tc_fence_before();
+        ok = __syncthreads_and(ok ? 1 : 0) != 0;
+        if (!ok) break;
+        if (tid == 0) {
+            tc::tma_store_2d(&map_y, (b0 + j) * 64, lt.t0, tile);
+            tc::bulk_commit();
+            const int32_t n = j + S - 1;          // next block to request: into the stage used by block j - 1
+            if (n < nblk) {
+                tc::bulk_wait_read<1>();          // that stage's store has finished reading shared memory
+                issue_load(n);
+            }
+        }
+    }
+    if (tid == 0) {
+        tc::bulk_wait_read<0>();
+        if (!ok) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tc::tmem_dealloc(tmem, C::TMEM_COLS);
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side: tensor maps and launches
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor [rows, cols] with a row pitch in elements; box = 64 columns x 128 rows
+static bool make_map_2d(CUtensorMap *m, const void *base, int64_t rows, int64_t cols, int64_t ld) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)TC_ROWS};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// 3-D view of one target's matrices in the pool: [slot][r_max rows][d columns]; box = 64 x box_rows x 1
+static bool make_map_3d(CUtensorMap *m, const void *base, int64_t d, int64_t r_max, int64_t slots,
+                        int64_t slot_stride, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)r_max, (cuuint64_t)slots};
+    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)slot_stride * 2};
+    cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int RP>
+static lora_status_t launch_tc_bucket(lora_pool_t *pool, const TcParams &P, const ApplyParams &AP,
+                                      int32_t units, cudaStream_t stream) {
+    CUtensorMap mx, myb, my, ma, mb;
+    const __nv_bfloat16 *w = pool->weights_dev;
+    if (!make_map_2d(&mx, AP.x, AP.T, AP.tv.d_in, AP.ldx) || !make_map_2d(&myb, AP.yb, AP.T, AP.tv.d_out, AP.ldyb) ||
+        !make_map_2d(&my, AP.y, AP.T, AP.tv.d_out, AP.ldy) ||
+        !make_map_3d(&ma, w + AP.tv.off_a, AP.tv.d_in, pool->r_max, pool->num_slots, pool->slot_stride, RP) ||
+        !make_map_3d(&mb, w + AP.tv.off_b, AP.tv.d_out, pool->r_max, pool->num_slots, pool->slot_stride, RP))
+        return LORA_ERR_INVALID_ARG;
+
+    constexpr int SH_SMEM = SH_STAGES * (XT_BYTES + ((RP * 128 + 1023) & ~1023)) + 256 + 1024;
+    static bool attr_done = false;
+    if (!attr_done) {
+        LORA_CUDA_TRY(cudaFuncSetAttribute(tc_shrink_kernel<RP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           SH_SMEM));
+        LORA_CUDA_TRY(cudaFuncSetAttribute(tc_expand_kernel<RP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           ExpandCfg<RP>::SMEM));
+        attr_done = true;
+    }
+    tc_shrink_kernel<RP><<<dim3(units, P.KS), TC_THREADS, SH_SMEM, stream>>>(P, mx, ma);
+    lora_status_t s = count_launch();
+    if (s != LORA_OK) return s;
+    tc_expand_kernel<RP><<<dim3(units, P.NS), TC_THREADS, ExpandCfg<RP>::SMEM, stream>>>(P, mb, myb, my);
+    return count_launch();
+}
+
+// Runs the long tiles of a batch.  Returns LORA_OK with *handled = false when the path does not
+// apply (no tensor-map support, misaligned operands); the caller then gives every tile to the
+// fused kernel.
+lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, void *workspace,
+                                   size_t workspace_bytes, cudaStream_t stream, bool *handled) {
+    *handled = false;
+    if (!AP.meta || AP.tile_m != TC_ROWS || AP.T < TC_ROWS) return LORA_OK;
+    if (!encode_fn()) return LORA_OK;
+    // TMA wants 16-byte aligned bases and row pitches
+    if ((((uintptr_t)AP.x | (uintptr_t)AP.yb | (uintptr_t)AP.y) & 15) || (AP.ldx % 8) || (AP.ldyb % 8) ||
+        (AP.ldy % 8))
+        return LORA_OK;
+    const int32_t RS = rank_bucket(pool->r_max);
+    const int32_t max_long = AP.T / TC_ROWS;
+    int32_t KS = next_pow2((2 * pool->sm_count + max_long - 1) / max_long);
+    if (KS > 8) KS = 8;
+    const int32_t nkb = (AP.tv.d_in + 63) / 64;
+    while (KS > 1 && KS > nkb) KS >>= 1;
+    const size_t per_split = (size_t)AP.T * RS * sizeof(float);
+    while (KS > 1 && per_split * KS > workspace_bytes) KS >>= 1;
+    if (!workspace || per_split * KS > workspace_bytes || ((uintptr_t)workspace & 15)) return LORA_OK;
+    int32_t NS = (4 * pool->sm_count + max_long - 1) / max_long;
+    const int32_t nblk = (AP.tv.d_out + 63) / 64;
+    if (NS > nblk) NS = nblk;
+    if (NS < 1) NS = 1;
+
+    TcParams P;
+    P.pool = AP.pool;
+    P.tv = AP.tv;
+    P.meta = AP.meta;
+    P.ws = (float *)workspace;
+    P.T = AP.T;
+    P.RS = RS;
+    P.KS = KS;
+    P.NS = NS;
+    const MetaLayout L = meta_layout(AP.T, AP.meta_slots, AP.tile_m);
+    if (L.words > 0x7fffffff) return LORA_OK;
+    P.moff_perm = (int32_t)L.perm;
+    P.moff_desc = (int32_t)L.tile_desc;
+    P.target_rows = pool->r_max;
+    const int32_t units = L.cap_tile;
+
+    lora_status_t s = LORA_OK;
+    if (pool->bucket_mask & 3u) s = launch_tc_bucket<16>(pool, P, AP, units, stream);
+    if (s == LORA_OK && (pool->bucket_mask & 4u)) s = launch_tc_bucket<32>(pool, P, AP, units, stream);
+    if (s == LORA_OK && (pool->bucket_mask & 8u)) s = launch_tc_bucket<64>(pool, P, AP, units, stream);
+    if (s == LORA_OK) *handled = true;
+    return s;
+}
+
+}  // namespace lora

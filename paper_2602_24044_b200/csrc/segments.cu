@@ -120,10 +120,12 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
             meta[L.tile_seg + idx] = seg;
             meta[L.tile_row0 + idx] = r0;
             meta[L.tile_rows + idx] = rows;
-            meta[L.tile_flags + idx] = (perm[r0 + rows - 1] - perm[r0] + 1 == rows) ? 1 : 0;
+            const int32_t contiguous = (perm[r0 + rows - 1] - perm[r0] + 1 == rows) ? 1 : 0;
+            meta[L.tile_flags + idx] = contiguous;
             const SlotEntry e = pool.table[s];
+            // private record: slot, position, rows (bits 0-14) | consecutive ids (bit 15) | rank, scale
             *reinterpret_cast<int4 *>(meta + L.tile_desc + 4 * (int64_t)idx) =
-                make_int4(s, r0, rows | (e.rank << 16), __float_as_int(e.scale));
+                make_int4(s, r0, rows | (contiguous << 15) | (e.rank << 16), __float_as_int(e.scale));
         }
     }
 
