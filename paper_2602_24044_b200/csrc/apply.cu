@@ -53,6 +53,8 @@ void fill_apply_params(lora_pool_t *pool, ApplyParams &P, int32_t target, const 
     P.rows_cap = 16;
     P.off_part = P.off_vst = P.off_stage = 0;
     P.path_filter = 0;
+    P.sub = 1;
+    P.aux = 1;
 }
 
 static lora_status_t apply_common(lora_pool_t *pool, int32_t target, const void *x, int64_t ldx,
@@ -72,7 +74,7 @@ static lora_status_t apply_common(lora_pool_t *pool, int32_t target, const void 
         bool handled = false;
         lora_status_t s = launch_tc_long_tiles(pool, P, workspace, workspace_bytes, stream, &handled);
         if (s != LORA_OK) return s;
-        P.path_filter = handled ? 1 : 0;
+        P.path_filter = handled ? 32 : 0;   // runs of >= 32 consecutive tokens were taken there
     }
     return launch_fused(pool, P, stream);
 }

@@ -29,6 +29,7 @@ struct ApplyParams {
     int32_t off_vpart, off_vh, off_vl;   // block partial of v, and v as bf16 high / low parts
     int32_t moff_perm, moff_desc, moff_tperm;   // word offsets of perm, tile records, tile row ids
     int32_t aux;               // this launch also counts invalid tokens and copies adapter-less rows
+    int32_t sub;               // fused path: 16-row pieces per tile (1 when tile_m <= 16)
     int32_t mrows;             // rows of an MMA row tile that can be occupied: 8 or 16
     int32_t xbufs;             // x stages: 1, or 2 when a tile spans several row tiles
     int32_t path_filter;       // 0 = every tile, 1 = skip tiles taken by the tensor-core kernel

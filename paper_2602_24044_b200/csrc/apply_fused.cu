@@ -426,23 +426,29 @@ fused_kernel(const ApplyParams P) {
     uint32_t ph[4] = {0u, 0u, 0u, 0u};
     int32_t n_tile = P.meta ? 0x7fffffff : P.T;
     // The grid holds as many clusters as fit on the GPU at once; each takes units cid, cid + G, ...
-    for (int32_t unit = cid; unit < P.units && unit < n_tile; unit += G) {
+    // Tiles of more than 16 rows are worked on in pieces of 16 rows (P.sub pieces per tile), so
+    // the shared-memory footprint of a block does not grow with tile_m.
+    const int32_t sub = P.sub, piece_rows = sub > 1 ? 16 : P.tile_m;
+    for (int32_t unit = cid; unit < P.units * sub && unit / sub < n_tile; unit += G) {
         // the tile record, the tile's row ids and (first time) the tile count are fetched side by
         // side, no load depends on another
         Tile tl;
         if (P.meta) {
-            if (tid < P.tile_m) rowidx[tid] = __ldg(P.meta + P.moff_tperm + unit * P.tile_m + tid);
+            const int32_t u = unit / sub, piece = unit - u * sub;
+            if (tid < piece_rows)
+                rowidx[tid] = __ldg(P.meta + P.moff_tperm + u * P.tile_m + piece * 16 + tid);
             if (unit == cid) n_tile = __ldg(P.meta + H_NTILE);
-            const int4 d = __ldg(reinterpret_cast<const int4 *>(P.meta + P.moff_desc) + unit);
+            const int4 d = __ldg(reinterpret_cast<const int4 *>(P.meta + P.moff_desc) + u);
+            const int32_t tile_rows = d.z & 0x7fff;
             tl.slot = d.x;
-            tl.row0 = d.y;
-            tl.rows = d.z & 0x7fff;
+            tl.row0 = d.y + piece * 16;
+            tl.rows = min(piece_rows, tile_rows - piece * 16);
             tl.rank = d.z >> 16;
             tl.scale = __int_as_float(d.w);
             tl.valid = d.x >= 0;
-            if (unit >= n_tile) break;
-            // full tiles of consecutive tokens belong to the tensor-core kernels when those ran
-            if (P.path_filter && tl.rows == 128 && ((d.z >> 15) & 1)) {
+            if (u >= n_tile) break;
+            // runs of consecutive tokens belong to the tensor-core kernels when those ran
+            if (tl.rows <= 0 || (P.path_filter && tile_rows >= P.path_filter && ((d.z >> 15) & 1))) {
                 __syncthreads();
                 continue;
             }
@@ -536,7 +542,7 @@ static lora_status_t launch_bucket(lora_pool_t *pool, ApplyParams P, int32_t C, 
                     RP, 8 * H, smem, C, n);
     }
     cfg.numAttrs = n_attrs;
-    int32_t want = P.units;   // tile units, or 16-row copy steps if there are more of those
+    int32_t want = P.units * P.sub;   // tile pieces, or 16-row copy steps if there are more of those
     if (P.aux && P.meta && !P.in_place && (P.T + 15) / 16 > want) want = (P.T + 15) / 16;
     int32_t G = occ_clusters > 0 && occ_clusters < want ? occ_clusters : want;
     if (pool->tuning[3] > 0 && pool->tuning[3] < G) G = pool->tuning[3];
@@ -547,9 +553,10 @@ static lora_status_t launch_bucket(lora_pool_t *pool, ApplyParams P, int32_t C, 
 
 lora_status_t launch_fused(lora_pool_t *pool, ApplyParams &P, cudaStream_t stream) {
     const int32_t tile_m = P.meta ? P.tile_m : 1;
-    P.rows_cap = (tile_m + 15) & ~15;
+    P.sub = tile_m > 16 ? (tile_m + 15) / 16 : 1;   // larger tiles are worked on in 16-row pieces
+    P.rows_cap = 16;
     P.mrows = tile_m <= 8 ? 8 : 16;
-    P.xbufs = tile_m > 16 ? 2 : 1;
+    P.xbufs = 1;
     P.moff_perm = P.moff_desc = P.moff_tperm = 0;
     if (P.meta) {
         const MetaLayout L = meta_layout(P.T, P.meta_slots, P.tile_m);
@@ -563,7 +570,7 @@ lora_status_t launch_fused(lora_pool_t *pool, ApplyParams &P, cudaStream_t strea
     if (C != 1 && C != 2 && C != 4 && C != 8) {
         C = 8;
         while (C > 1 && (P.tv.d_in / C < 256 || P.tv.d_out / C < 128)) C >>= 1;
-        while (C > 1 && (int64_t)P.units * C > (int64_t)16 * pool->sm_count) C >>= 1;
+        while (C > 1 && (int64_t)P.units * P.sub * C > (int64_t)64 * pool->sm_count) C >>= 1;
     }
     // one launch per rank bucket that has ever been loaded into the pool (ranks <= 16 share one)
     bool need[3] = {(pool->bucket_mask & 3u) != 0, (pool->bucket_mask & 4u) != 0,

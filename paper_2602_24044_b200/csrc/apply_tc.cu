@@ -166,24 +166,26 @@ struct TcParams {
     int32_t T, RS, KS, NS;
     int32_t moff_perm, moff_desc;
     int32_t target_rows;    // r_max: rows of a slot's matrices
+    __nv_bfloat16 *y;       // output, for tiles with fewer than 128 rows (stored row by row)
+    int64_t ldy;
 };
 
 // tile record -> (valid long tile of this bucket?, slot, first token, position in perm, rank, scale)
+constexpr int TC_MIN_ROWS = 32;    // shortest run of consecutive tokens given to the tensor cores
 struct LongTile {
-    int32_t slot, t0, row0, rank;
+    int32_t slot, t0, row0, rank, rows;
     float scale;
     bool ok;
 };
-__device__ __forceinline__ LongTile long_tile(const TcParams &P, int32_t unit, int32_t bucket) {
+__device__ __forceinline__ LongTile long_tile(const TcParams &P, int32_t unit) {
     LongTile lt;
     lt.ok = false;
     const int32_t n_tile = __ldg(P.meta + H_NTILE);
     if (unit >= n_tile) return lt;
     const int4 d = __ldg(reinterpret_cast<const int4 *>(P.meta + P.moff_desc) + unit);
     const int32_t rows = d.z & 0x7fff, contiguous = (d.z >> 15) & 1, rank = d.z >> 16;
-    if (d.x < 0 || rows != TC_ROWS || !contiguous) return lt;
-    const int32_t b = rank_bucket(rank);
-    if ((b <= 16 ? 16 : b) != bucket) return lt;
+    if (d.x < 0 || rows < TC_MIN_ROWS || !contiguous) return lt;
+    lt.rows = rows;
     lt.slot = d.x;
     lt.row0 = d.y;
     lt.rank = rank;
@@ -213,7 +215,7 @@ tc_shrink_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_x,
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(done + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const LongTile lt = long_tile(P, blockIdx.x, RP);
+    const LongTile lt = long_tile(P, blockIdx.x);
     if (!lt.ok) return;
     const int32_t ks = blockIdx.y;
     // K-blocks of 64 columns owned by this block
@@ -281,16 +283,18 @@ tc_shrink_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_x,
 #pragma unroll
         for (int c = 0; c < RP; c += 16) {
             uint32_t r[16];
-            if (nkb > 0) {
+            if (nkb > 0) {      // whole warps take part in the tensor-memory load
                 tc::tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + c, r);
                 tc::tmem_ld_wait();
             } else {
 #pragma unroll
                 for (int i = 0; i < 16; ++i) r[i] = 0u;
             }
+            if (m < lt.rows) {  // rows past a short tile's end belong to other tiles
 #pragma unroll
-            for (int i = 0; i < 16; i += 4)
-                *reinterpret_cast<uint4 *>(dst + c + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+                for (int i = 0; i < 16; i += 4)
+                    *reinterpret_cast<uint4 *>(dst + c + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+            }
         }
     } else if (tid == 0) {
         atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
@@ -331,7 +335,7 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(mma_done + S);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const LongTile lt = long_tile(P, blockIdx.x, RP);
+    const LongTile lt = long_tile(P, blockIdx.x);
     if (!lt.ok) return;
     // 64-column blocks of d_out owned by this block
     const int32_t nblk_all = (P.tv.d_out + 63) / 64;
@@ -360,7 +364,7 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
             float v[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) v[e] = 0.0f;
-            for (int32_t q = 0; q < P.KS; ++q) {
+            for (int32_t q = 0; q < P.KS && m < lt.rows; ++q) {   // rows past a short tile's end stay zero
                 const float4 a = *reinterpret_cast<const float4 *>(src + q * ks_stride + kg * 8);
                 const float4 b = *reinterpret_cast<const float4 *>(src + q * ks_stride + kg * 8 + 4);
                 v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
@@ -446,8 +450,20 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
         tc::tc_fence_before();
         ok = __syncthreads_and(ok ? 1 : 0) != 0;
         if (!ok) break;
+        if (lt.rows < TC_ROWS) {
+            // short tile: the rows after it belong to other tokens, so each thread stores its own row
+            const int32_t colb = (b0 + j) * 64;
+            if (m < lt.rows) {
+                __nv_bfloat16 *yrow = P.y + (int64_t)(lt.t0 + m) * P.ldy + colb;
+#pragma unroll
+                for (int chunk = 0; chunk < 8; ++chunk)
+                    if (colb + chunk * 8 < P.tv.d_out)
+                        *reinterpret_cast<uint4 *>(yrow + chunk * 8) =
+                            *reinterpret_cast<const uint4 *>(tile + m * 128 + ((chunk ^ (m & 7)) << 4));
+            }
+        }
         if (tid == 0) {
-            tc::tma_store_2d(&map_y, (b0 + j) * 64, lt.t0, tile);
+            if (lt.rows == TC_ROWS) tc::tma_store_2d(&map_y, (b0 + j) * 64, lt.t0, tile);
             tc::bulk_commit();
             const int32_t n = j + S - 1;          // next block to request: into the stage used by block j - 1
             if (n < nblk) {
@@ -554,8 +570,10 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
     if ((((uintptr_t)AP.x | (uintptr_t)AP.yb | (uintptr_t)AP.y) & 15) || (AP.ldx % 8) || (AP.ldyb % 8) ||
         (AP.ldy % 8))
         return LORA_OK;
-    const int32_t RS = rank_bucket(pool->r_max);
-    const int32_t max_long = AP.T / TC_ROWS;
+    const int32_t RS = rank_bucket(pool->r_max) < 16 ? 16 : rank_bucket(pool->r_max);
+    const int32_t max_long = (AP.T + TC_MIN_ROWS - 1) / TC_MIN_ROWS < AP.T / TC_ROWS + AP.meta_slots
+                                 ? (AP.T + TC_MIN_ROWS - 1) / TC_MIN_ROWS
+                                 : AP.T / TC_ROWS + AP.meta_slots;   // bound on tiles this path takes
     int32_t KS = next_pow2((2 * pool->sm_count + max_long - 1) / max_long);
     if (KS > 8) KS = 8;
     const int32_t nkb = (AP.tv.d_in + 63) / 64;
@@ -584,10 +602,13 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
     P.target_rows = pool->r_max;
     const int32_t units = L.cap_tile;
 
-    lora_status_t s = LORA_OK;
-    if (pool->bucket_mask & 3u) s = launch_tc_bucket<16>(pool, P, AP, units, stream);
-    if (s == LORA_OK && (pool->bucket_mask & 4u)) s = launch_tc_bucket<32>(pool, P, AP, units, stream);
-    if (s == LORA_OK && (pool->bucket_mask & 8u)) s = launch_tc_bucket<64>(pool, P, AP, units, stream);
+    P.y = AP.y;
+    P.ldy = AP.ldy;
+    // one pair of launches for every rank: the kernels are sized for the pool's largest rank
+    // bucket, and the rows above a slot's rank are zero
+    lora_status_t s = RS <= 16   ? launch_tc_bucket<16>(pool, P, AP, units, stream)
+                      : RS == 32 ? launch_tc_bucket<32>(pool, P, AP, units, stream)
+                                 : launch_tc_bucket<64>(pool, P, AP, units, stream);
     if (s == LORA_OK) *handled = true;
     return s;
 }

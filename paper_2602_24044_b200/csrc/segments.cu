@@ -45,9 +45,14 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
         for (int32_t t = tid; t < T; t += SEG_THREADS) tok[t] = slot_idx_g[t];
     const int32_t *slot_idx = staged ? tok : slot_idx_g;
     __syncthreads();
-    for (int32_t t = tid; t < T; t += SEG_THREADS) {
-        const int32_t s = slot_idx[t];
-        if (s >= 0 && s < N && occ[s]) atomicAdd(&cnt[s], 1);
+    // one shared-memory atomic per distinct slot per warp step: prefill batches are long runs of
+    // one slot, which would otherwise serialise on a single counter
+    for (int32_t base = warp * 32; base < T; base += SEG_THREADS) {
+        const int32_t t = base + lane;
+        const int32_t s = t < T ? slot_idx[t] : -1;
+        const bool act = s >= 0 && s < N && occ[s];
+        const uint32_t peers = __match_any_sync(0xffffffffu, act ? s : N + lane);
+        if (act && lane == __ffs(peers) - 1) atomicAdd(&cnt[s], __popc(peers));
     }
     __syncthreads();
 
@@ -92,17 +97,27 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
         if (n == 0) continue;
         const int32_t p0 = start[s], seg = segid[s];
         int32_t run = 0;
-        for (int32_t base = 0; base < T && run < n; base += 32) {
-            const int32_t t = base + lane;
-            const bool hit = t < T && slot_idx[t] == s;
-            const uint32_t m = __ballot_sync(0xffffffffu, hit);
-            if (hit) {
-                const int32_t j = run + __popc(m & ((1u << lane) - 1u));
-                perm[p0 + j] = t;
-                // private copy laid out by tile: tile k of the batch starts at k * tile_m
-                meta[L.tile_perm + (int64_t)tile0[s] * tile_m + j] = t;
+        // 128 tokens per step: the four loads are independent, the ballots keep token order
+        for (int32_t base = 0; base < T && run < n; base += 128) {
+            int32_t sv[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int32_t t = base + q * 32 + lane;
+                sv[q] = t < T ? slot_idx[t] : -2;
             }
-            run += __popc(m);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int32_t t = base + q * 32 + lane;
+                const bool hit = sv[q] == s;
+                const uint32_t m = __ballot_sync(0xffffffffu, hit);
+                if (hit) {
+                    const int32_t j = run + __popc(m & ((1u << lane) - 1u));
+                    perm[p0 + j] = t;
+                    // private copy laid out by tile: tile k of the batch starts at k * tile_m
+                    meta[L.tile_perm + (int64_t)tile0[s] * tile_m + j] = t;
+                }
+                run += __popc(m);
+            }
         }
         __syncwarp();
         const int32_t first = perm[p0], last = perm[p0 + n - 1];
@@ -183,12 +198,15 @@ lora_status_t launch_build_segments(lora_pool_t *pool, const int32_t *slot_idx_d
     int grid = (N + SEG_WARPS - 1) / SEG_WARPS;
     if (grid > 2 * pool->sm_count) grid = 2 * pool->sm_count;
     if (grid < 1) grid = 1;
-    const int32_t staged = T <= 8192 ? 1 : 0;   // the token list fits beside the per-slot arrays
+    // the token list is copied to shared memory when it fits beside the per-slot arrays
+    const int32_t staged = sizeof(int32_t) * (5 * (size_t)N + (size_t)T) <= 200 * 1024 ? 1 : 0;
     const size_t smem = sizeof(int32_t) * (5 * (size_t)N + (staged ? (size_t)T : 0));
-    if (smem > 48 * 1024) {
+    static size_t attr_smem = 48 * 1024;
+    if (smem > attr_smem) {
         cudaError_t e = cudaFuncSetAttribute(build_segments_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return cuda_fail(e);
+        attr_smem = smem;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
