@@ -27,7 +27,7 @@ struct ApplyParams {
     int32_t rows_cap;          // rows a unit can have, rounded up to 16
     int32_t off_part, off_vst, off_stage, off_x;
     int32_t off_vpart, off_vh, off_vl;   // block partial of v, and v as bf16 high / low parts
-    int32_t moff_perm, moff_desc, moff_tperm;   // word offsets of perm, tile records, tile row ids
+    int32_t moff_perm, moff_desc, moff_tperm, moff_piece;   // word offsets: perm, tile records, tile row ids, pieces
     int32_t aux;               // this launch also counts invalid tokens and copies adapter-less rows
     int32_t sub;               // fused path: 16-row pieces per tile (1 when tile_m <= 16)
     int32_t mrows;             // rows of an MMA row tile that can be occupied: 8 or 16

@@ -428,16 +428,24 @@ fused_kernel(const ApplyParams P) {
     // The grid holds as many clusters as fit on the GPU at once; each takes units cid, cid + G, ...
     // Tiles of more than 16 rows are worked on in pieces of 16 rows (P.sub pieces per tile), so
     // the shared-memory footprint of a block does not grow with tile_m.
+    // Such batches are walked through the metadata's list of pieces (no empty entries); decode
+    // batches (tile_m <= 16) index the tile table directly, which saves a dependent load.
     const int32_t sub = P.sub, piece_rows = sub > 1 ? 16 : P.tile_m;
-    for (int32_t unit = cid; unit < P.units * sub && unit / sub < n_tile; unit += G) {
-        // the tile record, the tile's row ids and (first time) the tile count are fetched side by
-        // side, no load depends on another
+    for (int32_t unit = cid; unit < P.units * sub && unit < n_tile; unit += G) {
+        // the tile record, the tile's row ids and (first time) the count are fetched side by side
         Tile tl;
         if (P.meta) {
-            const int32_t u = unit / sub, piece = unit - u * sub;
+            int32_t u = unit, piece = 0;
+            if (sub > 1) {
+                if (unit == cid) n_tile = __ldg(P.meta + H_NPIECE);   // here: number of pieces
+                if (unit >= n_tile) break;
+                const int32_t e = __ldg(P.meta + P.moff_piece + unit);
+                u = e >> 4;
+                piece = e & 15;
+            }
             if (tid < piece_rows)
                 rowidx[tid] = __ldg(P.meta + P.moff_tperm + u * P.tile_m + piece * 16 + tid);
-            if (unit == cid) n_tile = __ldg(P.meta + H_NTILE);
+            if (sub == 1 && unit == cid) n_tile = __ldg(P.meta + H_NTILE);
             const int4 d = __ldg(reinterpret_cast<const int4 *>(P.meta + P.moff_desc) + u);
             const int32_t tile_rows = d.z & 0x7fff;
             tl.slot = d.x;
@@ -446,7 +454,7 @@ fused_kernel(const ApplyParams P) {
             tl.rank = d.z >> 16;
             tl.scale = __int_as_float(d.w);
             tl.valid = d.x >= 0;
-            if (u >= n_tile) break;
+            if (sub == 1 && u >= n_tile) break;
             // runs of consecutive tokens belong to the tensor-core kernels when those ran
             if (tl.rows <= 0 || (P.path_filter && tile_rows >= P.path_filter && ((d.z >> 15) & 1))) {
                 __syncthreads();
@@ -557,20 +565,20 @@ lora_status_t launch_fused(lora_pool_t *pool, ApplyParams &P, cudaStream_t strea
     P.rows_cap = 16;
     P.mrows = tile_m <= 8 ? 8 : 16;
     P.xbufs = 1;
-    P.moff_perm = P.moff_desc = P.moff_tperm = 0;
+    P.moff_perm = P.moff_desc = P.moff_tperm = P.moff_piece = 0;
     if (P.meta) {
         const MetaLayout L = meta_layout(P.T, P.meta_slots, P.tile_m);
         if (L.words > 0x7fffffff) return LORA_ERR_SHAPE;
         P.moff_perm = (int32_t)L.perm;
         P.moff_desc = (int32_t)L.tile_desc;
         P.moff_tperm = (int32_t)L.tile_perm;
+        P.moff_piece = (int32_t)L.tile_piece;
     }
     // cluster size: as wide a split as the projection supports, narrower when there are many units
     int32_t C = pool->tuning[1];
     if (C != 1 && C != 2 && C != 4 && C != 8) {
         C = 8;
         while (C > 1 && (P.tv.d_in / C < 256 || P.tv.d_out / C < 128)) C >>= 1;
-        while (C > 1 && (int64_t)P.units * P.sub * C > (int64_t)64 * pool->sm_count) C >>= 1;
     }
     // one launch per rank bucket that has ever been loaded into the pool (ranks <= 16 share one)
     bool need[3] = {(pool->bucket_mask & 3u) != 0, (pool->bucket_mask & 4u) != 0,

@@ -67,12 +67,12 @@ struct TargetView {    // one adapted projection inside a slot
 // ---------------------------------------------------------------------------------------------
 enum { META_HEADER_WORDS = 16 };
 enum { H_T = 0, H_NACTIVE = 1, H_NINVALID = 2, H_NSEG = 3, H_NTILE = 4, H_TILE_M = 5,
-       H_LONG_MIN = 6, H_NSLOTS = 7, H_CAP_SEG = 8, H_CAP_TILE = 9 };
+       H_LONG_MIN = 6, H_NSLOTS = 7, H_CAP_SEG = 8, H_CAP_TILE = 9, H_NPIECE = 10 /* private */ };
 
 struct MetaLayout {
     int32_t cap_seg, cap_tile;
     int64_t perm, seg_slot, seg_start, seg_rank, seg_flags, tile_seg, tile_row0, tile_rows,
-        tile_flags, tile_desc, tile_perm, words;
+        tile_flags, tile_desc, tile_perm, tile_piece, words;
 };
 
 __host__ __device__ inline MetaLayout meta_layout(int32_t T, int32_t num_slots, int32_t tile_m) {
@@ -92,6 +92,8 @@ __host__ __device__ inline MetaLayout meta_layout(int32_t T, int32_t num_slots, 
     o = (o + 3) & ~(int64_t)3;            // library-private part, 16-byte aligned records
     L.tile_desc = o;  o += 4 * (int64_t)L.cap_tile;   // {slot, row0, rows | rank << 16, scale bits}
     L.tile_perm = o;  o += (int64_t)L.cap_tile * tile_m;   // tile k's token ids at k * tile_m
+    // 16-row pieces of all tiles, in tile order: (tile << 4) | piece; header word H_NPIECE counts them
+    L.tile_piece = o; o += (int64_t)L.cap_tile * ((tile_m + 15) / 16);
     L.words = o;
     return L;
 }

@@ -23,9 +23,10 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
     int32_t *segid = start + N;    // [N] segment number
     int32_t *tile0 = segid + N;    // [N] first tile number
     int32_t *occ = tile0 + N;      // [N] slot occupied (copy of the slot table's flag)
-    int32_t *tok = occ + N;        // [T] copy of the token list (only when `staged`)
-    __shared__ int32_t warp_tot[3][SEG_WARPS];
-    __shared__ int32_t totals[3];
+    int32_t *piece0 = occ + N;     // [N] first 16-row piece number
+    int32_t *tok = piece0 + N;     // [T] copy of the token list (only when `staged`)
+    __shared__ int32_t warp_tot[4][SEG_WARPS];
+    __shared__ int32_t totals[4];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const MetaLayout L = meta_layout(T, N, tile_m);
@@ -59,36 +60,49 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
     // ---- 2. exclusive prefix sums over slots: positions, segment numbers, tile numbers ------
     const int32_t per = (N + SEG_THREADS - 1) / SEG_THREADS;
     const int32_t lo = min(tid * per, N), hi = min(lo + per, N);
-    int32_t c = 0, z = 0, tl = 0;
+    // 16-row pieces of a segment of n tokens: full tiles have ppt pieces, the last tile fewer
+    const int32_t ppt = (tile_m + 15) / 16;
+    auto pieces_of = [&](int32_t n) {
+        return (n / tile_m) * ppt + ((n % tile_m) + 15) / 16;
+    };
+    int32_t c = 0, z = 0, tl = 0, pc = 0;
     for (int32_t s = lo; s < hi; ++s) {
         c += cnt[s];
         z += cnt[s] > 0;
         tl += (cnt[s] + tile_m - 1) / tile_m;
+        pc += pieces_of(cnt[s]);
     }
-    int32_t ic = c, iz = z, it = tl;   // inclusive warp scans
+    int32_t ic = c, iz = z, it = tl, ip = pc;   // inclusive warp scans
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const int32_t a = __shfl_up_sync(0xffffffffu, ic, o);
         const int32_t b = __shfl_up_sync(0xffffffffu, iz, o);
         const int32_t d = __shfl_up_sync(0xffffffffu, it, o);
-        if (lane >= o) { ic += a; iz += b; it += d; }
+        const int32_t e = __shfl_up_sync(0xffffffffu, ip, o);
+        if (lane >= o) { ic += a; iz += b; it += d; ip += e; }
     }
-    if (lane == 31) { warp_tot[0][warp] = ic; warp_tot[1][warp] = iz; warp_tot[2][warp] = it; }
+    if (lane == 31) {
+        warp_tot[0][warp] = ic; warp_tot[1][warp] = iz; warp_tot[2][warp] = it; warp_tot[3][warp] = ip;
+    }
     __syncthreads();
-    int32_t bc = 0, bz = 0, bt = 0;
-    for (int w = 0; w < warp; ++w) { bc += warp_tot[0][w]; bz += warp_tot[1][w]; bt += warp_tot[2][w]; }
-    int32_t rc = bc + ic - c, rz = bz + iz - z, rt = bt + it - tl;
+    int32_t bc = 0, bz = 0, bt = 0, bp = 0;
+    for (int w = 0; w < warp; ++w) {
+        bc += warp_tot[0][w]; bz += warp_tot[1][w]; bt += warp_tot[2][w]; bp += warp_tot[3][w];
+    }
+    int32_t rc = bc + ic - c, rz = bz + iz - z, rt = bt + it - tl, rp = bp + ip - pc;
     for (int32_t s = lo; s < hi; ++s) {
         start[s] = rc;
         segid[s] = rz;
         tile0[s] = rt;
+        piece0[s] = rp;
         rc += cnt[s];
         rz += cnt[s] > 0;
         rt += (cnt[s] + tile_m - 1) / tile_m;
+        rp += pieces_of(cnt[s]);
     }
-    if (tid == SEG_THREADS - 1) { totals[0] = rc; totals[1] = rz; totals[2] = rt; }
+    if (tid == SEG_THREADS - 1) { totals[0] = rc; totals[1] = rz; totals[2] = rt; totals[3] = rp; }
     __syncthreads();
-    const int32_t n_active = totals[0], n_seg = totals[1], n_tile = totals[2];
+    const int32_t n_active = totals[0], n_seg = totals[1], n_tile = totals[2], n_piece = totals[3];
 
     int32_t *perm = meta + L.perm;
     // ---- 3. one warp per occupied slot: write its run of perm, its segment and its tiles ----
@@ -141,6 +155,9 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
             // private record: slot, position, rows (bits 0-14) | consecutive ids (bit 15) | rank, scale
             *reinterpret_cast<int4 *>(meta + L.tile_desc + 4 * (int64_t)idx) =
                 make_int4(s, r0, rows | (contiguous << 15) | (e.rank << 16), __float_as_int(e.scale));
+            // private list of 16-row pieces (all earlier tiles of the segment are full)
+            for (int32_t i = 0; i < (rows + 15) / 16; ++i)
+                meta[L.tile_piece + piece0[s] + k * ppt + i] = (idx << 4) | i;
         }
     }
 
@@ -169,7 +186,8 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
             meta[H_NSLOTS] = N;
             meta[H_CAP_SEG] = L.cap_seg;
             meta[H_CAP_TILE] = L.cap_tile;
-            for (int i = H_CAP_TILE + 1; i < META_HEADER_WORDS; ++i) meta[i] = 0;
+            meta[H_NPIECE] = n_piece;
+            for (int i = H_NPIECE + 1; i < META_HEADER_WORDS; ++i) meta[i] = 0;
             meta[L.seg_start + n_seg] = n_active;
             if (n_invalid) atomicAdd(&pool.status[STATUS_INVALID_TOKENS], n_invalid);
         }
@@ -199,8 +217,8 @@ lora_status_t launch_build_segments(lora_pool_t *pool, const int32_t *slot_idx_d
     if (grid > 2 * pool->sm_count) grid = 2 * pool->sm_count;
     if (grid < 1) grid = 1;
     // the token list is copied to shared memory when it fits beside the per-slot arrays
-    const int32_t staged = sizeof(int32_t) * (5 * (size_t)N + (size_t)T) <= 200 * 1024 ? 1 : 0;
-    const size_t smem = sizeof(int32_t) * (5 * (size_t)N + (staged ? (size_t)T : 0));
+    const int32_t staged = sizeof(int32_t) * (6 * (size_t)N + (size_t)T) <= 200 * 1024 ? 1 : 0;
+    const size_t smem = sizeof(int32_t) * (6 * (size_t)N + (staged ? (size_t)T : 0));
     static size_t attr_smem = 48 * 1024;
     if (smem > attr_smem) {
         cudaError_t e = cudaFuncSetAttribute(build_segments_kernel,

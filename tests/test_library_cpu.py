@@ -84,6 +84,7 @@ def test_segments_bytes_matches_documented_layout():
     words = (words + 3) // 4 * 4 + 4 * cap_tile          # library-private tile records
     desc_end = words
     words += cap_tile * tile_m                           # library-private per-tile row ids
+    words += cap_tile * ((tile_m + 15) // 16)            # library-private list of 16-row pieces
     assert lb.segments_bytes(T, N, tile_m) == 4 * words
     assert lb.segments_bytes(0, N, tile_m) == 4 * 20
     with pytest.raises(lb.LoraError):
