@@ -158,8 +158,9 @@ lora_status_t lora_pool_set_tuning(lora_pool_t *pool, int32_t key, int32_t value
  *   tile_seg[cap_tile], tile_row0[cap_tile], tile_rows[cap_tile]
  *                each segment cut into pieces of at most tile_m rows (positions in perm)
  *   tile_flags[cap_tile]   bit0: the tile's tokens are consecutive ids
- *   (then, from the next 16-byte boundary, words private to the library: a 4-word record and
- *    tile_m row ids per tile; lora_segments_bytes counts them)
+ *   (then, from the next 16-byte boundary, words private to the library: a 4-word record per
+ *    tile, and a 4-word record plus 16 row ids per piece of at most 16 rows of a tile;
+ *    lora_segments_bytes counts them)
  * Unused entries are -1.  A token is active iff its slot id names an occupied slot; a token
  * that is neither active nor -1 is invalid (counted in header and in the pool's status word 0).
  * The result is an exact integer function of its inputs.

@@ -50,11 +50,10 @@ void fill_apply_params(lora_pool_t *pool, ApplyParams &P, int32_t target, const 
     P.in_place = (y == yb);
     P.units = meta ? meta_layout(T, pool->num_slots, tile_m).cap_tile : T;
     if (P.units < 1) P.units = 1;
-    P.rows_cap = 16;
-    P.off_part = P.off_vst = P.off_stage = 0;
+    P.off_part = P.off_vpart = P.off_vh = P.off_vl = P.off_stage = 0;
+    P.stage_bytes = P.n_stages = 0;
+    P.moff_perm = P.moff_udesc = P.moff_uperm = 0;
     P.path_filter = 0;
-    P.sub = 1;
-    P.aux = 1;
 }
 
 static lora_status_t apply_common(lora_pool_t *pool, int32_t target, const void *x, int64_t ldx,

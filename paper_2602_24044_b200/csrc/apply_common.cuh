@@ -20,19 +20,14 @@ struct ApplyParams {
     const int32_t *meta;       // grouped mode (nullptr = per-token mode)
     float *ws;                 // two-phase path: [KS][T][RS] fp32 partial v
     int32_t T, RS, KS, JS;
-    int32_t units;             // units (tiles or tokens) the grid covers
+    int32_t units;             // capacity of the unit list (tiles, 16-row pieces or tokens)
     int32_t tile_m, meta_slots;
     int32_t in_place;
     // fused path: shared-memory carve-up (bytes from the start of dynamic shared memory)
-    int32_t rows_cap;          // rows a unit can have, rounded up to 16
-    int32_t off_part, off_vst, off_stage, off_x;
-    int32_t off_vpart, off_vh, off_vl;   // block partial of v, and v as bf16 high / low parts
-    int32_t moff_perm, moff_desc, moff_tperm, moff_piece;   // word offsets: perm, tile records, tile row ids, pieces
-    int32_t aux;               // this launch also counts invalid tokens and copies adapter-less rows
-    int32_t sub;               // fused path: 16-row pieces per tile (1 when tile_m <= 16)
-    int32_t mrows;             // rows of an MMA row tile that can be occupied: 8 or 16
-    int32_t xbufs;             // x stages: 1, or 2 when a tile spans several row tiles
-    int32_t path_filter;       // 0 = every tile, 1 = skip tiles taken by the tensor-core kernel
+    int32_t off_part, off_vpart, off_vh, off_vl;   // warp partials, block partial, v as bf16 high / low parts
+    int32_t off_stage, stage_bytes, n_stages;      // ring of job buffers
+    int32_t moff_perm, moff_udesc, moff_uperm;     // word offsets: perm, unit records, unit row ids
+    int32_t path_filter;       // 0 = every unit; else skip runs of at least this many consecutive tokens
 };
 
 struct Tile {

@@ -1,23 +1,30 @@
-// Fused LoRA forward y = y_base + s_i * (x . A_i) . B_i (paper Section 2.2) in ONE launch.
+// Fused LoRA forward y = y_base + s_i * (x . A_i) . B_i (paper Section 2.2) in ONE launch for
+// every rank of a batch.
 //
-// A thread-block cluster owns one unit (a row tile of one adapter, or one token).  Block c of
-// the cluster takes the c-th slice of d_in for the shrink phase and the c-th slice of d_out for
-// the expand phase:
-//   1. everything the block will read is requested before any arithmetic: the A_i and B_i slices
-//      and the tile's x rows by bulk asynchronous copies into shared memory (mbarrier-signalled),
-//      the y_base rows by loads into registers; none of the expand operands depends on the shrink
-//      result, so their latency hides behind it;
-//   2. shrink: partial v over the block's d_in slice, split-K over the four warps, bf16 tensor-core
-//      MMA with fp32 accumulation;
-//   3. the partials are exchanged through distributed shared memory and summed in block order,
-//      identically in every block (no global workspace, no float atomics);
-//   4. expand over the block's d_out slice on the tensor cores, v carried as the sum of two bf16
-//      numbers (high and low part) so that it keeps ~16 mantissa bits; scale and residual add fused,
-//      one rounding to bf16 at the store.
-// Blocks are small (128 threads, ~44 KB of shared memory for decode tiles) so that many are
-// resident per SM: a decode batch fits on the GPU in one wave and the hardware overlaps their
-// latencies.  Every per-row sum is taken in a fixed order that does not depend on which other
-// rows share the tile (MMA rows are independent), so a row's result depends only on its inputs.
+// A unit is at most 16 token rows of one adapter.  A thread-block cluster owns one unit at a time
+// (units cid, cid + G, ... of the batch); block c of the cluster takes the c-th slice of d_in for
+// the shrink phase and the c-th slice of d_out for the expand phase.  Inside a block the work of
+// all its units is ONE stream of jobs
+//     unit 0: shrink chunk 0 .. na-1, expand chunk 0 .. nb-1, unit 1: shrink chunk 0 ...
+// and a job is one column chunk: the rank rows of A_i (or B_i), fetched by ONE tiled bulk copy
+// (TMA, 128-byte swizzle, the matrix viewed as blocks of 64 columns), plus the unit's rows of x (or
+// y_base), one bulk copy per row, into one stage of a small ring of shared-memory buffers
+// (mbarrier-signalled).  Few large copies matter: every bulk copy costs the issuing thread and the
+// copy engine a fixed time, and a copy per weight row made that time the bottleneck.  Warp 0 keeps the ring full: whenever a stage has been consumed it
+// requests the next job of the stream, which may belong to the next unit, so the memory latency of
+// a unit hides behind the arithmetic of the one before.  The chunk width shrinks as the rank
+// grows (256 / 128 / 64 columns for ranks <= 16 / 32 / 64), so a stage is the same size for
+// every rank and one launch serves all of them.
+//
+//   shrink  partial v over the block's d_in slice, split-K over the four warps, bf16 tensor-core
+//           MMA (m16n8k16) with fp32 accumulation carried across chunks in registers;
+//   exchange the block partials are summed through distributed shared memory in block order,
+//           identically in every block (no global workspace, no float atomics);
+//   expand  over the block's d_out slice on the tensor cores, v carried as the sum of two bf16
+//           numbers (high and low part, ~16 mantissa bits); scale and residual add fused, y_base
+//           read from the job's stage, one rounding to bf16 at the store.
+// Every per-row sum is taken in a fixed order that does not depend on which other rows share the
+// unit (MMA rows are independent), so a row's result depends only on its inputs.
 #include <cstdio>
 #include <cstdlib>
 
@@ -25,7 +32,18 @@
 
 namespace lora {
 
-constexpr int FT = 128;   // threads per block of the fused kernel
+constexpr int FT = 128;          // threads per block
+constexpr int UNIT_RING = 4;     // unit records held in shared memory: previous, current, next, next but one
+constexpr int RING_ENTRY = 80;   // one record: 16 bytes + 16 row ids
+constexpr int SM_RING = 64;      // byte offset of the record ring (mbarriers come first)
+constexpr int SM_HEADER = 384;   // bytes before the first carved-up buffer
+constexpr int MAX_STAGES = 4;
+constexpr int W_BYTES = 8192;    // weight tile of a job: rank bucket x chunk width x 2 bytes, for every bucket
+
+// tensor maps of one target: index rows / 8 - 1 for loads of `rows` rank rows (8, 16, .. 64)
+struct FusedMaps {
+    CUtensorMap a[8], b[8];
+};
 #ifndef LORA_FUSED_MIN_BLOCKS
 #define LORA_FUSED_MIN_BLOCKS 5   // resident blocks per SM the register budget is held to
 #endif
@@ -41,6 +59,9 @@ __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
 }
 __device__ __forceinline__ void fence_mbar_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
@@ -72,8 +93,14 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t by
         "l"(src), "r"(bytes), "r"(smem_u32(bar))
         : "memory");
 }
-__device__ __forceinline__ void prefetch_l2(const void *p) {
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+// one tile of a 4-D tensor (column in block, rank row, column block, slot) -> shared memory
+__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, int c0, int c1, int c2,
+                                            int c3, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, "
+        "%3, %4, %5}], [%6];" ::"r"(smem_u32(dst)),
+        "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar))
+        : "memory");
 }
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -115,7 +142,7 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t add
                  : "r"(addr));
 }
 // programmatic dependent launch: let the next kernel of the stream be scheduled / wait until all
-// work queued before this kernel is complete and visible (a no-op without the launch attribute)
+// work queued before this kernel is complete and visible (no-ops without the launch attribute)
 __device__ __forceinline__ void griddep_launch_dependents() {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
@@ -125,179 +152,235 @@ __device__ __forceinline__ void griddep_wait() {
 __device__ __forceinline__ uint32_t lds32(const __nv_bfloat16 *p) {
     return *reinterpret_cast<const uint32_t *>(p);
 }
-
-enum { BAR_A = 0, BAR_B = 1, BAR_X0 = 2, BAR_X1 = 3 };
-
-// One warp requests `nrows` rows of `ncols` bf16 each; row r comes from src + r * src_pitch (or
-// src + idx[r] * src_pitch) and lands at stage + r * pitch.
-__device__ __forceinline__ void issue_rows(uint64_t *bar, __nv_bfloat16 *stage, int pitch, int nrows,
-                                           int ncols, int lane, const __nv_bfloat16 *src,
-                                           int64_t src_pitch, const int32_t *idx) {
-    if (lane == 0) mbar_expect_tx(bar, (uint32_t)nrows * (uint32_t)ncols * 2u);
-    __syncwarp();
-    for (int r = lane; r < nrows; r += 32)
-        bulk_g2s(stage + r * pitch, src + (int64_t)(idx ? idx[r] : r) * src_pitch,
-                 (uint32_t)ncols * 2u, bar);
+__device__ __forceinline__ uint32_t lds32b(const unsigned char *p) {
+    return *reinterpret_cast<const uint32_t *>(p);
+}
+__device__ __forceinline__ int4 ldg_int4(const int32_t *p) {
+    int4 v;
+    asm volatile("ld.global.nc.v4.s32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ int32_t ldg_int(const int32_t *p) {
+    int32_t v;
+    asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
 }
 
-// RP: rank bucket (16, 32, 64); DCA / DCB: columns of A / B staged at a time.
-// H: 1 when a row tile holds at most 8 rows (decode tiles), 2 when rows 8..15 can be occupied.
-template <int RP, int DCA, int DCB, int H>
-__device__ __forceinline__ void fused_body(const ApplyParams &P, const Tile &tl, unsigned char *smem,
-                                           uint32_t crank, uint32_t csize, uint32_t (&ph)[4]) {
-    constexpr int PA = DCA + 8, PB = DCB + 8;   // shared-memory row pitches: +16 B against bank conflicts
-    constexpr int PV = RP + 8;                  // pitch of the bf16 copies of v
-    constexpr int NT_S = RP / 8;                // rank tiles of 8 in the shrink MMA
-    constexpr int KW = DCA / 4, NW = DCB / 4;   // columns per warp: shrink (split-K), expand
-    constexpr int NPASS = NW / 64;              // expand passes of 64 columns per warp
-    constexpr int A_BYTES = RP * PA * 2;
-    static_assert(NPASS >= 1 && KW % 16 == 0, "mapping");
+// ---------------------------------------------------------------------------------------------
+// units and the record ring
+// ---------------------------------------------------------------------------------------------
+struct Unit {
+    int32_t slot, rank, rows;
+    int32_t RP, CW;      // rank bucket (16, 32, 64) and its chunk width (256, 128, 64 columns)
+    int32_t rb;          // rank rows a tile load fetches: the rank rounded up to 8
+    int32_t na, nb;      // shrink / expand jobs of this block
+    float scale;
+    bool run;            // the unit has jobs in this launch
+};
 
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem);
-    const int32_t *rowidx = reinterpret_cast<const int32_t *>(smem + 64);
-    float *part = reinterpret_cast<float *>(smem + P.off_part);     // [4 warps][mrows][RP]
-    float *vpart = reinterpret_cast<float *>(smem + P.off_vpart);   // [rows][RP], read by the peers
-    __nv_bfloat16 *Vh = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_vh);   // [rows][PV]
-    __nv_bfloat16 *Vl = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_vl);
-    __nv_bfloat16 *As = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_stage);            // [RP][PA]
-    __nv_bfloat16 *Bs = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_stage + A_BYTES);  // [RP][PB]
-    __nv_bfloat16 *Xs = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_x);   // [xbufs][mrows][520]
-    constexpr int PX = 520;
+// record: {slot (-1: token without adapter, -2: past the end), position, rows | tile rows << 8 |
+// consecutive ids << 16 | rank << 17, scale bits}
+__device__ __forceinline__ Unit decode_unit(const ApplyParams &P, const int4 rec, int32_t a_w,
+                                            int32_t b_w) {
+    Unit u;
+    u.slot = rec.x;
+    u.rows = rec.z & 0xff;
+    const int32_t tile_rows = (rec.z >> 8) & 0xff, contiguous = (rec.z >> 16) & 1;
+    u.rank = (rec.z >> 17) & 0x7f;
+    u.scale = __int_as_float(rec.w);
+    // runs of consecutive tokens belong to the tensor-core kernels when those ran
+    u.run = rec.x >= 0 && u.rows > 0 && u.rank > 0 &&
+            !(P.path_filter && contiguous && tile_rows >= P.path_filter);
+    const int32_t sh = u.rank <= 16 ? 0 : u.rank <= 32 ? 1 : 2;
+    u.rb = (u.rank + 7) & ~7;
+    u.RP = 16 << sh;
+    u.CW = 256 >> sh;
+    u.na = (a_w + u.CW - 1) >> (8 - sh);
+    u.nb = (b_w + u.CW - 1) >> (8 - sh);
+    return u;
+}
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-    const int32_t d_in = P.tv.d_in, d_out = P.tv.d_out, rows = tl.rows, rank = tl.rank;
-    const int32_t rank16 = (rank + 15) & ~15;
-    constexpr int32_t mrows = 8 * H;
-    constexpr bool hi_rows = H == 2;   // rows 8..15 of a row tile can be occupied
-    const int32_t n_mt = (rows + 15) >> 4;
-    const __nv_bfloat16 *A = P.pool.weights + (int64_t)tl.slot * P.pool.slot_stride + P.tv.off_a;
-    const __nv_bfloat16 *B = P.pool.weights + (int64_t)tl.slot * P.pool.slot_stride + P.tv.off_b;
+struct UnitRegs {   // a record on its way from global memory to the ring (lane 16: record, lanes 0-15: row ids)
+    int4 rec;
+    int32_t rowid;
+};
 
-    // this block's column slices (multiples of 8 columns)
-    const int32_t Wa = (d_in + (int32_t)csize * 8 - 1) / ((int32_t)csize * 8) * 8;
-    const int32_t a_lo = min((int32_t)crank * Wa, d_in), a_hi = min(a_lo + Wa, d_in);
-    const int32_t na = (a_hi - a_lo + DCA - 1) / DCA;
-    const int32_t Wb = (d_out + (int32_t)csize * 8 - 1) / ((int32_t)csize * 8) * 8;
-    const int32_t b_lo = min((int32_t)crank * Wb, d_out), b_hi = min(b_lo + Wb, d_out);
-    const int32_t nb = (b_hi - b_lo + DCB - 1) / DCB;
-    const int32_t n_items = na * n_mt;   // (column chunk, row tile) pairs of the shrink phase
-
-    auto issue_x = [&](int32_t it, int buf) {
-        const int32_t c = it / n_mt, mt = it - c * n_mt;
-        const int32_t col0 = a_lo + c * DCA;
-        issue_rows(&bars[BAR_X0 + buf], Xs + buf * mrows * PX, PX, min(mrows, rows - mt * 16),
-                   min(DCA, a_hi - col0), lane, P.x + col0, P.ldx, rowidx + mt * 16);
-    };
-    // y_base of one (chunk, row tile, pass) in the MMA accumulator layout: [column tile of 8][row
-    // g / g+8], two adjacent columns (2t, 2t+1) per word
-    auto load_yb = [&](uint32_t (&ybw)[8][H], int32_t c, int32_t mt, int p) {
-        const int32_t col0 = b_lo + c * DCB, ncols = min(DCB, b_hi - col0);
-#pragma unroll
-        for (int h = 0; h < H; ++h) {
-            const int32_t m = mt * 16 + g + 8 * h;
-            const __nv_bfloat16 *row = P.yb + (int64_t)rowidx[m < rows ? m : 0] * P.ldyb + col0 + 2 * t;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int32_t col = warp * NW + p * 64 + j * 8;
-                ybw[j][h] = 0u;
-                if (m < rows && col < ncols)
-                    ybw[j][h] = __ldg(reinterpret_cast<const uint32_t *>(row + col));
+// Requests the record of unit u.  `cap` bounds the addresses that may be read; whether u is a real
+// unit is decided when the record is stored.
+__device__ __forceinline__ UnitRegs fetch_unit(const ApplyParams &P, int32_t u, int32_t cap, int lane) {
+    UnitRegs m;
+    m.rec = make_int4(-2, 0, 0, 0);
+    m.rowid = 0;
+    if (u >= cap) return m;
+    if (P.meta) {
+        if (lane == 16) m.rec = ldg_int4(P.meta + P.moff_udesc + 4 * (int64_t)u);
+        else if (lane < 16) m.rowid = ldg_int(P.meta + P.moff_uperm + 16 * (int64_t)u + lane);
+    } else {
+        m.rowid = u;
+        if (lane == 16) {
+            const int32_t s = ldg_int(P.slot_idx + u);
+            m.rec = make_int4(-1, s != -1 ? 1 : 0, 0, 0);   // y = 1: not an adapter-less token either
+            if (s >= 0 && s < P.pool.num_slots) {
+                const SlotEntry e = P.pool.table[s];
+                if (e.loaded)
+                    m.rec = make_int4(s, u, 1 | (1 << 8) | (1 << 16) | (e.rank << 17),
+                                      __float_as_int(e.scale));
             }
         }
-    };
-
-    // ---- everything this block reads is requested here ------------------------------------------
-    if (warp == 0 && na > 0)
-        issue_rows(&bars[BAR_A], As, PA, rank, min(DCA, a_hi - a_lo), lane, A + a_lo, d_in, nullptr);
-    if (warp == 1 && nb > 0)
-        issue_rows(&bars[BAR_B], Bs, PB, rank, min(DCB, b_hi - b_lo), lane, B + b_lo, d_out, nullptr);
-    if (warp == 2 && n_items > 0) issue_x(0, 0);
-    if (warp == 3) {
-        // rows rank .. rank16-1 of the B stage are multiplied by zeros of v: make them finite
-        const int32_t vec_per_row = PB / 8;
-        for (int i = lane; i < (rank16 - rank) * vec_per_row; i += 32)
-            reinterpret_cast<uint4 *>(Bs + (rank + i / vec_per_row) * PB)[i % vec_per_row] =
-                make_uint4(0, 0, 0, 0);
     }
-    // y_base of the first row tile is requested into registers now (it is used last); for tiles
-    // with more row tiles the rest is pulled towards L2 (128-byte lines)
-    uint32_t ybw[NPASS][8][H];
-    if (nb > 0) load_yb(ybw[0], 0, 0, 0);
-    if (rows > 16 && b_hi > b_lo) {
-        const int32_t lines = ((b_hi - b_lo) * 2 + 127) >> 7;
-        for (int i = tid; i < (rows - 16) * lines; i += FT) {
-            const int m = 16 + i / lines, l = i % lines;
-            prefetch_l2(reinterpret_cast<const char *>(P.yb + (int64_t)rowidx[m] * P.ldyb + b_lo) +
-                        (l << 7));
+    return m;
+}
+__device__ __forceinline__ void store_unit(unsigned char *smem, int32_t iter, const UnitRegs &m,
+                                           bool real, int lane) {
+    unsigned char *e = smem + SM_RING + (iter % UNIT_RING) * RING_ENTRY;
+    if (lane == 16) *reinterpret_cast<int4 *>(e) = real ? m.rec : make_int4(-2, 0, 0, 0);
+    else if (lane < 16) reinterpret_cast<int32_t *>(e + 16)[lane] = m.rowid;
+}
+
+// What every part of a block needs to know about its place and progress.
+struct Ctx {
+    unsigned char *smem;
+    uint64_t *full;            // [n_stages] a job's data has landed
+    int32_t cid, G, n_units;   // cluster index, clusters in the grid, units in the batch
+    uint32_t crank, csize;
+    int32_t a_lo, a_hi, b_lo, b_hi;   // this block's column slices of d_in and d_out
+    int32_t ci;                // unit iteration the consumers work on
+    int32_t cq;                // jobs consumed so far
+    int32_t pi, pj, pq;        // producer: unit iteration, job within it, jobs requested so far
+    bool pending_wait;         // a cluster barrier arrive whose wait is still to come
+    bool ok;                   // no wait has expired
+};
+
+// Warp 0: request jobs until the ring is full.  Jobs of the unit after the current one may be
+// requested (their record is already in the ring); anything further ahead waits.
+__device__ __forceinline__ void issue_jobs(const ApplyParams &P, const FusedMaps &M, Ctx &cx, int lane) {
+    const int32_t S = P.n_stages;
+    while (cx.pq - cx.cq < S) {
+        Unit un;
+        const int32_t *rowidx;
+        for (;;) {
+            if (cx.pi > cx.ci + 1 || cx.cid + cx.pi * cx.G >= cx.n_units) return;
+            const unsigned char *e = cx.smem + SM_RING + (cx.pi % UNIT_RING) * RING_ENTRY;
+            un = decode_unit(P, *reinterpret_cast<const int4 *>(e), cx.a_hi - cx.a_lo, cx.b_hi - cx.b_lo);
+            rowidx = reinterpret_cast<const int32_t *>(e + 16);
+            if (un.run && cx.pj < un.na + un.nb) break;
+            ++cx.pi;
+            cx.pj = 0;
         }
+        const int st = cx.pq % S;
+        unsigned char *ws = cx.smem + P.off_stage + st * P.stage_bytes;
+        const bool shrink = cx.pj < un.na;
+        const int32_t c = shrink ? cx.pj : cx.pj - un.na;
+        const int32_t col0 = (shrink ? cx.a_lo : cx.b_lo) + c * un.CW;   // a multiple of 64
+        const int32_t ncols = min(un.CW, (shrink ? cx.a_hi : cx.b_hi) - col0);
+        const int32_t pitch = un.CW + 8;
+        const CUtensorMap *map = shrink ? &M.a[(un.rb >> 3) - 1] : &M.b[(un.rb >> 3) - 1];
+        const __nv_bfloat16 *tok = (shrink ? P.x : P.yb) + col0;
+        const int64_t tld = shrink ? P.ldx : P.ldyb;
+        __nv_bfloat16 *ts = reinterpret_cast<__nv_bfloat16 *>(ws + W_BYTES);
+        if (lane == 0) {
+            // the tile load always delivers its whole box: rb rows of CW columns
+            mbar_expect_tx(&cx.full[st], (uint32_t)un.rb * (uint32_t)un.CW * 2u +
+                                             (uint32_t)un.rows * (uint32_t)ncols * 2u);
+            tma_load_4d(ws, map, 0, 0, col0 >> 6, un.slot, &cx.full[st]);
+        }
+        __syncwarp();
+        if (lane < un.rows)
+            bulk_g2s(ts + lane * pitch, tok + (int64_t)rowidx[lane] * tld, (uint32_t)ncols * 2u,
+                     &cx.full[st]);
+        ++cx.pj;
+        ++cx.pq;
     }
+}
 
-    // mbarrier phase bits live across the units a block processes
-    uint32_t &ph_a = ph[BAR_A], &ph_b = ph[BAR_B], &ph_x0 = ph[BAR_X0], &ph_x1 = ph[BAR_X1];
-    bool ok = true;
+// All threads: wait for the data of the next job; returns its stage.
+__device__ __forceinline__ const unsigned char *acquire_job(const ApplyParams &P, Ctx &cx) {
+    const int st = cx.cq % P.n_stages;
+    cx.ok = mbar_wait(&cx.full[st], (uint32_t)(cx.cq / P.n_stages) & 1u) && cx.ok;
+    return cx.smem + P.off_stage + st * P.stage_bytes;
+}
+// All threads: the job's stage is free again; warp 0 refills the ring.
+__device__ __forceinline__ void release_job(const ApplyParams &P, const FusedMaps &M, Ctx &cx, int warp,
+                                            int lane) {
+    __syncthreads();
+    ++cx.cq;
+    if (warp == 0) issue_jobs(P, M, cx, lane);
+}
 
-    // ---- shrink: warp w takes columns [w*KW, (w+1)*KW) of the staged chunk (split-K) ------------
-    for (int32_t it = 0; it < n_items; ++it) {
-        const int32_t c = it / n_mt, mt = it - c * n_mt;
-        const int32_t ncols = min(DCA, a_hi - (a_lo + c * DCA));
-        if (mt == 0) {
-            if (c > 0 && warp == 0)
-                issue_rows(&bars[BAR_A], As, PA, rank, ncols, lane, A + a_lo + c * DCA, d_in, nullptr);
-            ok = mbar_wait(&bars[BAR_A], ph_a) && ok;
-            ph_a ^= 1;
-        }
-        int buf = 0;
-        if (P.xbufs == 2) {
-            buf = it & 1;
-            if (it + 1 < n_items && warp == 2) issue_x(it + 1, buf ^ 1);
-        } else if (it > 0 && warp == 2) {
-            issue_x(it, 0);
-        }
-        if (buf == 0) { ok = mbar_wait(&bars[BAR_X0], ph_x0) && ok; ph_x0 ^= 1; }
-        else { ok = mbar_wait(&bars[BAR_X1], ph_x1) && ok; ph_x1 ^= 1; }
+// RP: rank bucket of the unit; H: 1 when a unit holds at most 8 rows, 2 when rows 8..15 can be occupied.
+template <int RP, int H>
+__device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps &M, const Unit &un,
+                                          const int32_t *rowidx, Ctx &cx) {
+    constexpr int CW = 4096 / RP;      // columns per job
+    constexpr int PW = CW + 8;         // row pitch of the token rows: +16 B against bank conflicts
+    constexpr int PV = RP + 8;         // pitch of the bf16 copies of v
+    constexpr int NT_S = RP / 8;       // rank tiles of 8 in the shrink MMA
+    constexpr int KW = CW / 4;         // shrink: columns per warp and job (split-K)
+    constexpr int NW = CW / 4;         // expand: columns per warp and job
+    constexpr int NT_E = NW / 8;       // expand: column tiles of 8 per warp
+    constexpr int mrows = 8 * H;
+    constexpr bool hi_rows = H == 2;
 
-        const __nv_bfloat16 *X = Xs + buf * mrows * PX;
-        float acc[NT_S][4];
+    unsigned char *smem = cx.smem;
+    float *part = reinterpret_cast<float *>(smem + P.off_part);     // [4 warps][mrows][RP]
+    float *vpart = reinterpret_cast<float *>(smem + P.off_vpart);   // [mrows][RP], read by the peers
+    __nv_bfloat16 *Vh = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_vh);   // [mrows][PV]
+    __nv_bfloat16 *Vl = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_vl);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+    const int32_t rows = un.rows, rank = un.rank;
+    const int32_t rank16 = (rank + 15) & ~15;
+    // A weight tile is stored as blocks of 64 columns, rb rows of 128 bytes each, the 16-byte
+    // chunks of a row exchanged by the row number's low three bits (128-byte swizzle).
+    const uint32_t blk_bytes = (uint32_t)un.rb * 128u;
+
+    // ---- shrink: warp w takes columns [w*KW, (w+1)*KW) of every chunk (split-K) ------------------
+    float acc[NT_S][4];
 #pragma unroll
-        for (int nt = 0; nt < NT_S; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.0f;
+    for (int nt = 0; nt < NT_S; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.0f;
+    for (int32_t c = 0; c < un.na; ++c) {
+        const unsigned char *As = acquire_job(P, cx);   // tile of A_i, then [mrows][PW] rows of x
+        const __nv_bfloat16 *X = reinterpret_cast<const __nv_bfloat16 *>(As + W_BYTES);
+        const int32_t ncols = min(CW, cx.a_hi - (cx.a_lo + c * CW));
 #pragma unroll
         for (int ks = 0; ks < KW; ks += 16) {
             const int kk = warp * KW + ks;
             if (kk < ncols) {
                 const bool full = ncols - kk >= 16;   // else only 8 columns are left
                 uint32_t a[4];
-                a[0] = lds32(X + g * PX + kk + 2 * t);
-                a[1] = hi_rows ? lds32(X + (g + 8) * PX + kk + 2 * t) : 0u;
-                a[2] = full ? lds32(X + g * PX + kk + 8 + 2 * t) : 0u;
-                a[3] = (full && hi_rows) ? lds32(X + (g + 8) * PX + kk + 8 + 2 * t) : 0u;
+                a[0] = lds32(X + g * PW + kk + 2 * t);
+                a[1] = hi_rows ? lds32(X + (g + 8) * PW + kk + 2 * t) : 0u;
+                a[2] = full ? lds32(X + g * PW + kk + 8 + 2 * t) : 0u;
+                a[3] = (full && hi_rows) ? lds32(X + (g + 8) * PW + kk + 8 + 2 * t) : 0u;
+                const unsigned char *ab = As + (uint32_t)(kk >> 6) * blk_bytes + g * 128 + 4 * t;
+                const uint32_t ch = (uint32_t)(kk & 63) >> 3;   // even
 #pragma unroll
-                for (int nt = 0; nt < NT_S; ++nt) {
-                    const __nv_bfloat16 *ar = As + (nt * 8 + g) * PA + kk + 2 * t;
-                    mma16816(acc[nt], a, lds32(ar), full ? lds32(ar + 8) : 0u);
-                }
+                for (int nt = 0; nt < NT_S; ++nt)
+                    mma16816(acc[nt], a, lds32b(ab + nt * 1024 + ((ch ^ (uint32_t)g) << 4)),
+                             full ? lds32b(ab + nt * 1024 + (((ch + 1) ^ (uint32_t)g) << 4)) : 0u);
             }
         }
-#pragma unroll
-        for (int nt = 0; nt < NT_S; ++nt) {
-            float *p0 = part + (warp * mrows + g) * RP + nt * 8 + 2 * t;
-            *reinterpret_cast<float2 *>(p0) = make_float2(acc[nt][0], acc[nt][1]);
-            if (hi_rows) *reinterpret_cast<float2 *>(p0 + 8 * RP) = make_float2(acc[nt][2], acc[nt][3]);
-        }
-        __syncthreads();
-        // block partial: the four warps' sums in warp order, accumulated over column chunks
-        for (int i = tid; i < mrows * RP; i += FT) {
-            const int r = i / RP, k = i - r * RP;
-            if (mt * 16 + r < rows) {
-                const float s = ((part[(0 * mrows + r) * RP + k] + part[(1 * mrows + r) * RP + k]) +
-                                 part[(2 * mrows + r) * RP + k]) + part[(3 * mrows + r) * RP + k];
-                float *dst = vpart + (mt * 16 + r) * RP + k;
-                *dst = c == 0 ? s : *dst + s;
-            }
-        }
-        __syncthreads();   // partial buffers, the x stage and (after the last row tile) the A stage are free
+        release_job(P, M, cx, warp, lane);
     }
-    if (n_items == 0) {   // this block owns no d_in columns: its partial is zero
-        for (int i = tid; i < rows * RP; i += FT) vpart[i] = 0.0f;
+    // the peers have finished reading the previous unit's partial before it is overwritten
+    if (cx.pending_wait) {
+        cluster_wait();
+        cx.pending_wait = false;
+    }
+#pragma unroll
+    for (int nt = 0; nt < NT_S; ++nt) {
+        float *p0 = part + (warp * mrows + g) * RP + nt * 8 + 2 * t;
+        *reinterpret_cast<float2 *>(p0) = make_float2(acc[nt][0], acc[nt][1]);
+        if (hi_rows) *reinterpret_cast<float2 *>(p0 + 8 * RP) = make_float2(acc[nt][2], acc[nt][3]);
+    }
+    __syncthreads();
+    // block partial: the four warps' sums in warp order
+    for (int i = tid; i < mrows * RP; i += FT) {
+        const int r = i / RP;
+        if (r < rows)
+            vpart[i] = ((part[i] + part[mrows * RP + i]) + part[2 * mrows * RP + i]) + part[3 * mrows * RP + i];
     }
     // ---- exchange: every block sums all blocks' partials in block order -------------------------
     cluster_arrive();
@@ -313,7 +396,7 @@ __device__ __forceinline__ void fused_body(const ApplyParams &P, const Tile &tl,
                 float pv[8];
 #pragma unroll
                 for (uint32_t q = 0; q < 8; ++q)
-                    pv[q] = q < csize ? ld_peer_f32(vp_addr + (uint32_t)(m * RP + k) * 4u, q) : 0.0f;
+                    pv[q] = q < cx.csize ? ld_peer_f32(vp_addr + (uint32_t)(m * RP + k) * 4u, q) : 0.0f;
 #pragma unroll
                 for (uint32_t q = 0; q < 8; ++q) v += pv[q];
             }
@@ -322,196 +405,268 @@ __device__ __forceinline__ void fused_body(const ApplyParams &P, const Tile &tl,
             Vl[m * PV + k] = __float2bfloat16_rn(v - __bfloat162float(hi));
         }
     }
-    cluster_arrive();   // done reading the peers; the matching wait is at the end
+    cluster_arrive();   // done reading the peers; the matching wait comes before the next overwrite
+    cx.pending_wait = true;
     __syncthreads();
 
-    // ---- expand: warp w takes columns [w*NW, (w+1)*NW) of the staged chunk ----------------------
-    {
-        const float s = tl.scale;
-        for (int32_t c = 0; c < nb; ++c) {
-            const int32_t col0 = b_lo + c * DCB, ncols = min(DCB, b_hi - col0);
-            if (c > 0 && warp == 1)
-                issue_rows(&bars[BAR_B], Bs, PB, rank, ncols, lane, B + col0, d_out, nullptr);
-            ok = mbar_wait(&bars[BAR_B], ph_b) && ok;
-            ph_b ^= 1;
-            for (int32_t mt = 0; mt < n_mt; ++mt) {
-                const __nv_bfloat16 *vh = Vh + (mt * 16 + g) * PV + 2 * t;
-                const __nv_bfloat16 *vl = Vl + (mt * 16 + g) * PV + 2 * t;
+    // ---- expand: warp w takes columns [w*NW, (w+1)*NW) of every chunk ---------------------------
+    const float s = un.scale;
+    for (int32_t c = 0; c < un.nb; ++c) {
+        const unsigned char *Bs = acquire_job(P, cx);   // tile of B_i, then [mrows][PW] rows of y_base
+        const __nv_bfloat16 *Ys = reinterpret_cast<const __nv_bfloat16 *>(Bs + W_BYTES);
+        const int32_t col0 = cx.b_lo + c * CW, ncols = min(CW, cx.b_hi - col0);
+        const int base = warp * NW;
+        if (base < ncols) {
+            float ex[NT_E][4];
 #pragma unroll
-                for (int p = 0; p < NPASS; ++p) {
-                    const int base = warp * NW + p * 64;
-                    if (base >= ncols) continue;
-                    // y_base of the next pass is requested while this pass computes
-                    if (p == 0 && (c > 0 || mt > 0)) load_yb(ybw[0], c, mt, 0);
-                    if (p + 1 < NPASS) load_yb(ybw[(p + 1) % NPASS], c, mt, p + 1);
-                    float acc[8][4];
+            for (int j = 0; j < NT_E; ++j) ex[j][0] = ex[j][1] = ex[j][2] = ex[j][3] = 0.0f;
+            const __nv_bfloat16 *vh = Vh + g * PV + 2 * t;
+            const __nv_bfloat16 *vl = Vl + g * PV + 2 * t;
+            for (int ks = 0; ks < rank16; ks += 16) {
+                uint32_t ah[4], al[4];
+                ah[0] = lds32(vh + ks);
+                ah[1] = hi_rows ? lds32(vh + 8 * PV + ks) : 0u;
+                ah[2] = lds32(vh + ks + 8);
+                ah[3] = hi_rows ? lds32(vh + 8 * PV + ks + 8) : 0u;
+                al[0] = lds32(vl + ks);
+                al[1] = hi_rows ? lds32(vl + 8 * PV + ks) : 0u;
+                al[2] = lds32(vl + ks + 8);
+                al[3] = hi_rows ? lds32(vl + 8 * PV + ks + 8) : 0u;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.0f;
-                    for (int ks = 0; ks < rank16; ks += 16) {
-                        uint32_t ah[4], al[4];
-                        ah[0] = lds32(vh + ks);
-                        ah[1] = hi_rows ? lds32(vh + 8 * PV + ks) : 0u;
-                        ah[2] = lds32(vh + ks + 8);
-                        ah[3] = hi_rows ? lds32(vh + 8 * PV + ks + 8) : 0u;
-                        al[0] = lds32(vl + ks);
-                        al[1] = hi_rows ? lds32(vl + 8 * PV + ks) : 0u;
-                        al[2] = lds32(vl + ks + 8);
-                        al[3] = hi_rows ? lds32(vl + 8 * PV + ks + 8) : 0u;
+                for (int np = 0; np < NT_E / 2; ++np) {
+                    // matrices: (k 0..7, tile 2np), (k 8..15, tile 2np), (k 0..7, 2np+1), (k 8..15, 2np+1)
+                    const int mi = lane >> 3;
+                    const int col = base + (np * 2 + (mi >> 1)) * 8;
+                    const unsigned char *bp = Bs + (uint32_t)(col >> 6) * blk_bytes +
+                                              (ks + (mi & 1) * 8 + (lane & 7)) * 128 +
+                                              ((((uint32_t)(col & 63) >> 3) ^ (uint32_t)(lane & 7)) << 4);
+                    uint32_t b[4];
+                    ldmatrix_x4_trans(b, smem_u32(bp));
+                    mma16816(ex[np * 2], ah, b[0], b[1]);
+                    mma16816(ex[np * 2], al, b[0], b[1]);
+                    mma16816(ex[np * 2 + 1], ah, b[2], b[3]);
+                    mma16816(ex[np * 2 + 1], al, b[2], b[3]);
+                }
+            }
+            // epilogue straight from the accumulator layout: each lane owns two adjacent columns of
+            // a row per column tile; a quad covers 16 contiguous bytes
 #pragma unroll
-                        for (int np = 0; np < 4; ++np) {
-                            // matrices: (k 0..7, tile 2np), (k 8..15, tile 2np), (k 0..7, 2np+1), (k 8..15, 2np+1)
-                            const int mi = lane >> 3;
-                            const __nv_bfloat16 *bp = Bs + (ks + (mi & 1) * 8 + (lane & 7)) * PB + base +
-                                                      (np * 2 + (mi >> 1)) * 8;
-                            uint32_t b[4];
-                            ldmatrix_x4_trans(b, smem_u32(bp));
-                            mma16816(acc[np * 2], ah, b[0], b[1]);
-                            mma16816(acc[np * 2], al, b[0], b[1]);
-                            mma16816(acc[np * 2 + 1], ah, b[2], b[3]);
-                            mma16816(acc[np * 2 + 1], al, b[2], b[3]);
-                        }
-                    }
-                    // epilogue straight from the accumulator layout: each lane owns two adjacent
-                    // columns of a row per column tile; a quad covers 16 contiguous bytes
+            for (int h = 0; h < H; ++h) {
+                const int32_t m = g + 8 * h;
+                if (m < rows && cx.ok) {
+                    __nv_bfloat16 *yrow = P.y + (int64_t)rowidx[m] * P.ldy + col0 + base + 2 * t;
+                    const __nv_bfloat16 *ybrow = Ys + m * PW + base + 2 * t;
 #pragma unroll
-                    for (int h = 0; h < H; ++h) {
-                        const int32_t m = mt * 16 + g + 8 * h;
-                        if (m < rows && ok) {
-                            __nv_bfloat16 *yrow = P.y + (int64_t)rowidx[m] * P.ldy + col0 + base + 2 * t;
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                if (base + j * 8 < ncols) {
-                                    const uint32_t w = ybw[p][j][h];
-                                    const float y0 = fmaf(s, acc[j][2 * h], __uint_as_float(w << 16));
-                                    const float y1 = fmaf(s, acc[j][2 * h + 1], __uint_as_float(w & 0xffff0000u));
-                                    *reinterpret_cast<uint32_t *>(yrow + j * 8) = pack2(y0, y1);
-                                }
-                            }
+                    for (int j = 0; j < NT_E; ++j) {
+                        if (base + j * 8 < ncols) {
+                            const uint32_t w = lds32(ybrow + j * 8);
+                            const float y0 = fmaf(s, ex[j][2 * h], __uint_as_float(w << 16));
+                            const float y1 = fmaf(s, ex[j][2 * h + 1], __uint_as_float(w & 0xffff0000u));
+                            *reinterpret_cast<uint32_t *>(yrow + j * 8) = pack2(y0, y1);
                         }
                     }
                 }
             }
-            __syncthreads();   // the B stage is free
         }
+        release_job(P, M, cx, warp, lane);
     }
-    if (!ok && tid == 0) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
-    cluster_wait();   // no block leaves while a peer may still read its partials
 }
 
-// One kernel per rank bucket (RP) and row-tile occupancy (H); units of another bucket are skipped.
-// P.aux != 0 marks the launch that also counts invalid tokens and copies adapter-less rows.
-template <int RP, int DCA, int DCB, int H>
+// H: 1 when a unit holds at most 8 rows (decode tiles, single tokens), 2 otherwise.
+template <int H>
 __global__ void __launch_bounds__(FT, LORA_FUSED_MIN_BLOCKS)
-fused_kernel(const ApplyParams P) {
-    extern __shared__ __align__(128) unsigned char smem[];
-    const uint32_t csize = cluster_nctarank(), crank = cluster_ctarank();
-    const int32_t cid = (int32_t)(blockIdx.x / csize), G = (int32_t)(gridDim.x / csize);
-    const int tid = threadIdx.x;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem);
-    int32_t *rowidx = reinterpret_cast<int32_t *>(smem + 64);
+fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    Ctx cx;
+    cx.smem = smem;
+    cx.full = reinterpret_cast<uint64_t *>(smem);
+    cx.csize = cluster_nctarank();
+    cx.crank = cluster_ctarank();
+    cx.cid = (int32_t)(blockIdx.x / cx.csize);
+    cx.G = (int32_t)(gridDim.x / cx.csize);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // the swizzled tiles want 1024-byte aligned stages; the carve-up assumes an aligned base
+    if (smem_u32(smem) & 1023u) {
+        if (tid == 0 && blockIdx.x == 0) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
+        return;
+    }
 
-    // set-up that touches no global memory; the next kernel on the stream may be scheduled from
-    // here on, and this one waits for everything queued before it
+    // set-up that touches no global memory: barriers, and zeros in every stage (rows above a
+    // unit's rank are never copied, and what they hold is multiplied by zeros of v)
     if (tid == 0) {
-        mbar_init(&bars[BAR_A], 1);
-        mbar_init(&bars[BAR_B], 1);
-        mbar_init(&bars[BAR_X0], 1);
-        mbar_init(&bars[BAR_X1], 1);
+        for (int s = 0; s < P.n_stages; ++s) mbar_init(&cx.full[s], 1);
         fence_mbar_init();
     }
+    for (int i = tid; i < P.n_stages * P.stage_bytes / 16; i += FT)
+        reinterpret_cast<uint4 *>(smem + P.off_stage)[i] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async();   // the stages are written by bulk copies from here on
+    // the next kernel on the stream may be scheduled from here on, and this one waits for
+    // everything queued before it
     griddep_launch_dependents();
     __syncthreads();
     griddep_wait();
 
-    uint32_t ph[4] = {0u, 0u, 0u, 0u};
-    int32_t n_tile = P.meta ? 0x7fffffff : P.T;
-    // The grid holds as many clusters as fit on the GPU at once; each takes units cid, cid + G, ...
-    // Tiles of more than 16 rows are worked on in pieces of 16 rows (P.sub pieces per tile), so
-    // the shared-memory footprint of a block does not grow with tile_m.
-    // Such batches are walked through the metadata's list of pieces (no empty entries); decode
-    // batches (tile_m <= 16) index the tile table directly, which saves a dependent load.
-    const int32_t sub = P.sub, piece_rows = sub > 1 ? 16 : P.tile_m;
-    for (int32_t unit = cid; unit < P.units * sub && unit < n_tile; unit += G) {
-        // the tile record, the tile's row ids and (first time) the count are fetched side by side
-        Tile tl;
-        if (P.meta) {
-            int32_t u = unit, piece = 0;
-            if (sub > 1) {
-                if (unit == cid) n_tile = __ldg(P.meta + H_NPIECE);   // here: number of pieces
-                if (unit >= n_tile) break;
-                const int32_t e = __ldg(P.meta + P.moff_piece + unit);
-                u = e >> 4;
-                piece = e & 15;
-            }
-            if (tid < piece_rows)
-                rowidx[tid] = __ldg(P.meta + P.moff_tperm + u * P.tile_m + piece * 16 + tid);
-            if (sub == 1 && unit == cid) n_tile = __ldg(P.meta + H_NTILE);
-            const int4 d = __ldg(reinterpret_cast<const int4 *>(P.meta + P.moff_desc) + u);
-            const int32_t tile_rows = d.z & 0x7fff;
-            tl.slot = d.x;
-            tl.row0 = d.y + piece * 16;
-            tl.rows = min(piece_rows, tile_rows - piece * 16);
-            tl.rank = d.z >> 16;
-            tl.scale = __int_as_float(d.w);
-            tl.valid = d.x >= 0;
-            if (sub == 1 && u >= n_tile) break;
-            // runs of consecutive tokens belong to the tensor-core kernels when those ran
-            if (tl.rows <= 0 || (P.path_filter && tile_rows >= P.path_filter && ((d.z >> 15) & 1))) {
-                __syncthreads();
-                continue;
-            }
-        } else {
-            if (tid == 0) rowidx[0] = unit;
-            MetaLayout L;
-            tl = resolve_unit(P, L, unit);
-        }
-        __syncthreads();   // row ids visible
-        if (!tl.valid) {
-            if (!P.meta && P.aux) {   // per-token mode: this token has no adapter
-                if (crank == 0 && tid == 0 && P.slot_idx[unit] != -1)
-                    atomicAdd(&P.pool.status[STATUS_INVALID_TOKENS], 1);
-                if (!P.in_place) copy_rows(P, rowidx, 1, (int32_t)crank, (int32_t)csize);
-            }
-            __syncthreads();   // before the row ids are overwritten
-            continue;
-        }
-        const int32_t b = rank_bucket(tl.rank);
-        if ((b <= 16 ? 16 : b) != RP) {   // another launch's bucket
-            __syncthreads();
-            continue;
-        }
-        fused_body<RP, DCA, DCB, H>(P, tl, smem, crank, csize, ph);
+    // this block's column slices (multiples of 64 columns: tile loads address whole column blocks)
+    {
+        const int32_t cs64 = (int32_t)cx.csize * 64;
+        const int32_t Wa = (P.tv.d_in + cs64 - 1) / cs64 * 64, Wb = (P.tv.d_out + cs64 - 1) / cs64 * 64;
+        cx.a_lo = min((int32_t)cx.crank * Wa, P.tv.d_in);
+        cx.a_hi = min(cx.a_lo + Wa, P.tv.d_in);
+        cx.b_lo = min((int32_t)cx.crank * Wb, P.tv.d_out);
+        cx.b_hi = min(cx.b_lo + Wb, P.tv.d_out);
     }
+    // the number of units and the records of this cluster's first two units, side by side
+    {
+        UnitRegs m0, m1;
+        if (warp == 3) {
+            m0 = fetch_unit(P, cx.cid, P.units, lane);
+            m1 = fetch_unit(P, cx.cid + cx.G, P.units, lane);
+        }
+        cx.n_units = P.meta ? ldg_int(P.meta + H_NPIECE) : P.T;
+        if (cx.n_units > P.units) cx.n_units = P.units;
+        if (warp == 3) {
+            store_unit(smem, 0, m0, cx.cid < cx.n_units, lane);
+            store_unit(smem, 1, m1, cx.cid + cx.G < cx.n_units, lane);
+        }
+    }
+    __syncthreads();
+    cx.ci = 0;
+    cx.cq = cx.pq = cx.pi = cx.pj = 0;
+    cx.pending_wait = false;
+    cx.ok = true;
+
+    for (;; ++cx.ci) {
+        const int32_t u = cx.cid + cx.ci * cx.G;
+        if (u >= cx.n_units) break;
+        // the record of the unit after next is requested now and stored when this unit is done
+        UnitRegs mn;
+        if (warp == 3) mn = fetch_unit(P, u + 2 * cx.G, cx.n_units, lane);
+        const unsigned char *e = smem + SM_RING + (cx.ci % UNIT_RING) * RING_ENTRY;
+        const int4 rec = *reinterpret_cast<const int4 *>(e);
+        const int32_t *rowidx = reinterpret_cast<const int32_t *>(e + 16);
+        const Unit un = decode_unit(P, rec, cx.a_hi - cx.a_lo, cx.b_hi - cx.b_lo);
+        if (warp == 0) issue_jobs(P, M, cx, lane);
+        if (un.run) {
+            if (un.RP == 16) unit_body<16, H>(P, M, un, rowidx, cx);
+            else if (un.RP == 32) unit_body<32, H>(P, M, un, rowidx, cx);
+            else unit_body<64, H>(P, M, un, rowidx, cx);
+        } else if (!P.meta && rec.x == -1) {   // per-token mode: this token has no adapter
+            if (cx.crank == 0 && tid == 0 && rec.y) atomicAdd(&P.pool.status[STATUS_INVALID_TOKENS], 1);
+            if (!P.in_place) copy_rows(P, rowidx, 1, (int32_t)cx.crank, (int32_t)cx.csize);
+        }
+        if (warp == 3) store_unit(smem, cx.ci + 2, mn, true, lane);
+        __syncthreads();   // the new record is visible; nobody reads the current one any more
+    }
+    if (!cx.ok && tid == 0) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
+
     // rows that take no adapter: y_base -> y, 16 rows per cluster step (grouped mode, out of place)
-    if (P.meta && !P.in_place && P.aux) {
+    if (P.meta && !P.in_place) {
+        int32_t *rowidx = reinterpret_cast<int32_t *>(smem + SM_RING + 16);
         const int32_t n_active = __ldg(P.meta + H_NACTIVE);
-        for (int32_t first = cid * 16; first < P.T - n_active; first += G * 16) {
+        for (int32_t first = cx.cid * 16; first < P.T - n_active; first += cx.G * 16) {
             const int32_t rows = min(16, P.T - n_active - first);
             __syncthreads();
             if (tid < rows) rowidx[tid] = __ldg(P.meta + P.moff_perm + n_active + first + tid);
             __syncthreads();
-            copy_rows(P, rowidx, rows, (int32_t)crank, (int32_t)csize);
+            copy_rows(P, rowidx, rows, (int32_t)cx.crank, (int32_t)cx.csize);
         }
     }
+    // no block leaves while a peer may still read its partials
+    if (cx.pending_wait) cluster_wait();
 }
 
-// One launch for the tiles of one rank bucket.  The shared-memory carve-up is sized for that bucket.
-template <int RP, int DCA, int DCB, int H>
-static lora_status_t launch_bucket(lora_pool_t *pool, ApplyParams P, int32_t C, cudaStream_t stream) {
-    auto kern = fused_kernel<RP, DCA, DCB, H>;
-    const int32_t tile_m = P.meta ? P.tile_m : 1;
-    const int32_t vrows = H == 1 ? 8 : P.rows_cap;      // rows of the v buffers
-    int32_t o = (64 + P.rows_cap * 4 + 127) & ~127;     // mbarriers, row ids
-    P.off_part = o;   o += 4 * (8 * H) * RP * 4;
-    P.off_vpart = o;  o += vrows * RP * 4;
-    P.off_vh = o;     o += vrows * (RP + 8) * 2;
-    P.off_vl = o;     o += vrows * (RP + 8) * 2;
-    o = (o + 127) & ~127;
-    P.off_stage = o;  o += RP * (DCA + 8) * 2 + RP * (DCB + 8) * 2;
-    P.off_x = o;      o += P.xbufs * (8 * H) * 520 * 2;
-    P.off_vst = 0;
+// ---------------------------------------------------------------------------------------------
+// host side: tensor maps (built once per target, kept in the pool handle) and launch
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn tiled_encoder() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+// One target's matrix family in the pool, [slot][r_max rows][d columns], viewed as a 4-D tensor
+// (column inside a 64-column block, rank row, column block, slot); box = 64 x rows x blocks x 1.
+// The last column block of a row may reach into the next row (or, in the last row of the last
+// slot, into the pool's slack bytes); such columns are never used.
+static bool weight_map(CUtensorMap *m, const void *base, int64_t d, int64_t r_max, int64_t slots,
+                       int64_t slot_stride, int rows, int blocks) {
+    EncodeTiledFn fn = tiled_encoder();
+    if (!fn) return false;
+    cuuint64_t dims[4] = {64, (cuuint64_t)r_max, (cuuint64_t)((d + 63) / 64), (cuuint64_t)slots};
+    cuuint64_t strides[3] = {(cuuint64_t)d * 2, 128, (cuuint64_t)slot_stride * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)rows, (cuuint32_t)blocks, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static lora_status_t target_maps(lora_pool_t *pool, const ApplyParams &P, const FusedMaps **out) {
+    static_assert(sizeof(lora_pool::TargetMaps) == sizeof(FusedMaps), "same layout");
+    int32_t target = -1;
+    for (int32_t t = 0; t < pool->num_targets; ++t)
+        if (pool->target_views[t].off_a == P.tv.off_a) target = t;
+    if (target < 0) return LORA_ERR_INVALID_ARG;
+    if (pool->fused_maps.empty()) {
+        pool->fused_maps.resize(pool->num_targets);
+        pool->fused_maps_ready.assign(pool->num_targets, 0);
+    }
+    lora_pool::TargetMaps &tm = pool->fused_maps[target];
+    if (!pool->fused_maps_ready[target]) {
+        const __nv_bfloat16 *w = pool->weights_dev;
+        for (int i = 0; i < 8; ++i) {
+            const int rows = 8 * (i + 1);
+            if (rows > ((pool->r_max + 7) & ~7)) break;   // no slot holds that many rank rows
+            const int blocks = rows <= 16 ? 4 : rows <= 32 ? 2 : 1;   // chunk width 256 / 128 / 64
+            if (!weight_map(&tm.a[i], w + P.tv.off_a, P.tv.d_in, pool->r_max, pool->num_slots,
+                            pool->slot_stride, rows, blocks) ||
+                !weight_map(&tm.b[i], w + P.tv.off_b, P.tv.d_out, pool->r_max, pool->num_slots,
+                            pool->slot_stride, rows, blocks))
+                return cuda_fail(cudaErrorNotSupported);
+        }
+        pool->fused_maps_ready[target] = 1;
+    }
+    *out = reinterpret_cast<const FusedMaps *>(&tm);
+    return LORA_OK;
+}
+
+// Shared-memory carve-up and launch.  The buffers are sized for the largest rank bucket that has
+// ever been loaded into the pool.
+template <int H>
+static lora_status_t launch_h(lora_pool_t *pool, ApplyParams P, int32_t C, const FusedMaps *maps,
+                              cudaStream_t stream) {
+    auto kern = fused_kernel<H>;
+    const int32_t mrows = 8 * H;
+    const int32_t RPmax = (pool->bucket_mask & 8u) ? 64 : (pool->bucket_mask & 4u) ? 32 : 16;
+    // a stage: the weight tile, then the token rows at the widest chunk (rank bucket 16)
+    const int32_t stage = (W_BYTES + mrows * (256 + 8) * 2 + 1023) & ~1023;
+    int32_t S = pool->tuning[5];
+    if (S < 2 || S > MAX_STAGES) S = 3;
+    int32_t o = SM_HEADER;
+    P.off_part = o;   o += 4 * mrows * RPmax * 4;
+    P.off_vpart = o;  o += mrows * RPmax * 4;
+    P.off_vh = o;     o += mrows * (RPmax + 8) * 2;
+    P.off_vl = o;     o += mrows * (RPmax + 8) * 2;
+    o = (o + 1023) & ~1023;
+    P.off_stage = o;  o += S * stage;
+    P.stage_bytes = stage;
+    P.n_stages = S;
     const int32_t smem = o;
-    (void)tile_m;
 
     static int32_t attr_smem = 0;
     if (smem > attr_smem) {
@@ -546,61 +701,42 @@ static lora_status_t launch_bucket(lora_pool_t *pool, ApplyParams P, int32_t C, 
         }
         occ_smem = smem; occ_c = C; occ_clusters = n;
         if (getenv("LORA_B200_DEBUG"))
-            fprintf(stderr, "lora_b200: fused kernel rank<=%d rows<=%d: smem %d B, cluster %d, resident clusters %d\n",
-                    RP, 8 * H, smem, C, n);
+            fprintf(stderr, "lora_b200: fused kernel rows<=%d ranks<=%d: smem %d B (%d stages of %d B), cluster %d, "
+                    "resident clusters %d\n", mrows, RPmax, smem, S, stage, C, n);
     }
     cfg.numAttrs = n_attrs;
-    int32_t want = P.units * P.sub;   // tile pieces, or 16-row copy steps if there are more of those
-    if (P.aux && P.meta && !P.in_place && (P.T + 15) / 16 > want) want = (P.T + 15) / 16;
+    int32_t want = P.units;   // units, or 16-row copy steps if there are more of those
+    if (P.meta && !P.in_place && (P.T + 15) / 16 > want) want = (P.T + 15) / 16;
     int32_t G = occ_clusters > 0 && occ_clusters < want ? occ_clusters : want;
     if (pool->tuning[3] > 0 && pool->tuning[3] < G) G = pool->tuning[3];
     cfg.gridDim = dim3((unsigned)(G * C), 1, 1);
-    LORA_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, P));
+    LORA_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, P, *maps));
     return count_launch();
 }
 
 lora_status_t launch_fused(lora_pool_t *pool, ApplyParams &P, cudaStream_t stream) {
     const int32_t tile_m = P.meta ? P.tile_m : 1;
-    P.sub = tile_m > 16 ? (tile_m + 15) / 16 : 1;   // larger tiles are worked on in 16-row pieces
-    P.rows_cap = 16;
-    P.mrows = tile_m <= 8 ? 8 : 16;
-    P.xbufs = 1;
-    P.moff_perm = P.moff_desc = P.moff_tperm = P.moff_piece = 0;
+    P.moff_perm = P.moff_udesc = P.moff_uperm = 0;
+    P.units = P.T;
     if (P.meta) {
         const MetaLayout L = meta_layout(P.T, P.meta_slots, P.tile_m);
         if (L.words > 0x7fffffff) return LORA_ERR_SHAPE;
         P.moff_perm = (int32_t)L.perm;
-        P.moff_desc = (int32_t)L.tile_desc;
-        P.moff_tperm = (int32_t)L.tile_perm;
-        P.moff_piece = (int32_t)L.tile_piece;
+        P.moff_udesc = (int32_t)L.unit_desc;
+        P.moff_uperm = (int32_t)L.unit_perm;
+        P.units = L.cap_unit;
     }
-    // cluster size: as wide a split as the projection supports, narrower when there are many units
+    if (P.units < 1) P.units = 1;
+    // cluster size: as wide a split as the projection supports
     int32_t C = pool->tuning[1];
     if (C != 1 && C != 2 && C != 4 && C != 8) {
         C = 8;
         while (C > 1 && (P.tv.d_in / C < 256 || P.tv.d_out / C < 128)) C >>= 1;
     }
-    // one launch per rank bucket that has ever been loaded into the pool (ranks <= 16 share one)
-    bool need[3] = {(pool->bucket_mask & 3u) != 0, (pool->bucket_mask & 4u) != 0,
-                    (pool->bucket_mask & 8u) != 0};
-    if (!need[0] && !need[1] && !need[2]) need[0] = true;   // empty pool: rows are still copied
-    P.aux = 1;
-    for (int b = 0; b < 3; ++b) {
-        if (!need[b]) continue;
-        lora_status_t s;
-        if (P.mrows == 8) {
-            s = b == 0 ? launch_bucket<16, 512, 512, 1>(pool, P, C, stream)
-              : b == 1 ? launch_bucket<32, 256, 256, 1>(pool, P, C, stream)
-                       : launch_bucket<64, 256, 256, 1>(pool, P, C, stream);
-        } else {
-            s = b == 0 ? launch_bucket<16, 512, 512, 2>(pool, P, C, stream)
-              : b == 1 ? launch_bucket<32, 256, 256, 2>(pool, P, C, stream)
-                       : launch_bucket<64, 256, 256, 2>(pool, P, C, stream);
-        }
-        if (s != LORA_OK) return s;
-        P.aux = 0;
-    }
-    return LORA_OK;
+    const FusedMaps *maps = nullptr;
+    lora_status_t s = target_maps(pool, P, &maps);
+    if (s != LORA_OK) return s;
+    return tile_m <= 8 ? launch_h<1>(pool, P, C, maps, stream) : launch_h<2>(pool, P, C, maps, stream);
 }
 
 }  // namespace lora

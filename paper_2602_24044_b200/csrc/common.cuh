@@ -1,6 +1,7 @@
 // Shared declarations of the lora_b200 CUDA library (host handle, device views, metadata layout).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -72,7 +73,8 @@ enum { H_T = 0, H_NACTIVE = 1, H_NINVALID = 2, H_NSEG = 3, H_NTILE = 4, H_TILE_M
 struct MetaLayout {
     int32_t cap_seg, cap_tile;
     int64_t perm, seg_slot, seg_start, seg_rank, seg_flags, tile_seg, tile_row0, tile_rows,
-        tile_flags, tile_desc, tile_perm, tile_piece, words;
+        tile_flags, tile_desc, unit_desc, unit_perm, words;
+    int32_t cap_unit;
 };
 
 __host__ __device__ inline MetaLayout meta_layout(int32_t T, int32_t num_slots, int32_t tile_m) {
@@ -91,9 +93,13 @@ __host__ __device__ inline MetaLayout meta_layout(int32_t T, int32_t num_slots, 
     L.tile_flags = o; o += L.cap_tile;
     o = (o + 3) & ~(int64_t)3;            // library-private part, 16-byte aligned records
     L.tile_desc = o;  o += 4 * (int64_t)L.cap_tile;   // {slot, row0, rows | rank << 16, scale bits}
-    L.tile_perm = o;  o += (int64_t)L.cap_tile * tile_m;   // tile k's token ids at k * tile_m
-    // 16-row pieces of all tiles, in tile order: (tile << 4) | piece; header word H_NPIECE counts them
-    L.tile_piece = o; o += (int64_t)L.cap_tile * ((tile_m + 15) / 16);
+    // Units of the fused kernel: every tile cut into pieces of at most 16 rows, in tile order
+    // (a tile of tile_m <= 16 rows is one unit).  Header word H_NPIECE counts them.  One record
+    // per unit {slot, position in perm, rows | tile rows << 8 | consecutive ids << 16 | rank << 17,
+    // scale bits} and the unit's token ids at unit * 16.
+    L.cap_unit = L.cap_tile * ((tile_m + 15) / 16);
+    L.unit_desc = o;  o += 4 * (int64_t)L.cap_unit;
+    L.unit_perm = o;  o += 16 * (int64_t)L.cap_unit;
     L.words = o;
     return L;
 }
@@ -127,6 +133,13 @@ struct lora_pool {
     int32_t sm_count = 148;
     uint32_t bucket_mask = 0;           // rank buckets (8/16/32/64 -> bits 0..3) ever loaded into a slot
     int32_t tuning[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    // Tensor maps of the fused kernel, built on first use: per target, 8 for A and 8 for B (one
+    // per number of rank rows 8, 16, .. 64 a tile load fetches).
+    struct alignas(64) TargetMaps {
+        CUtensorMap a[8], b[8];
+    };
+    std::vector<TargetMaps> fused_maps;
+    std::vector<uint8_t> fused_maps_ready;
 
     // Shapes of the metadata tables built through this handle (the table itself lives on the
     // device; apply calls need T and tile_m on the host to size their grids).

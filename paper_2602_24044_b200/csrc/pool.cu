@@ -43,7 +43,9 @@ static PoolLayout pool_layout(const lora_pool_desc_t *d) {
     L.off_table = 256;
     L.off_staging = align_up(L.off_table + sizeof(SlotEntry) * (size_t)d->num_slots, 256);
     L.off_weights = align_up(L.off_staging + L.staging_elems * 2, 256);
-    L.bytes = L.off_weights + (size_t)L.slot_stride * 2 * (size_t)d->num_slots;
+    // 256 bytes of slack after the last slot: tiled loads of 64-column blocks may start inside
+    // the last row of the last matrix and run up to 126 bytes past its end
+    L.bytes = L.off_weights + (size_t)L.slot_stride * 2 * (size_t)d->num_slots + 256;
     return L;
 }
 

@@ -127,8 +127,9 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
                 if (hit) {
                     const int32_t j = run + __popc(m & ((1u << lane) - 1u));
                     perm[p0 + j] = t;
-                    // private copy laid out by tile: tile k of the batch starts at k * tile_m
-                    meta[L.tile_perm + (int64_t)tile0[s] * tile_m + j] = t;
+                    // private copy laid out by unit (16-row piece of a tile), 16 ids per unit
+                    const int32_t k = j / tile_m, jj = j - k * tile_m;
+                    meta[L.unit_perm + 16 * (int64_t)(piece0[s] + k * ppt + (jj >> 4)) + (jj & 15)] = t;
                 }
                 run += __popc(m);
             }
@@ -155,9 +156,13 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
             // private record: slot, position, rows (bits 0-14) | consecutive ids (bit 15) | rank, scale
             *reinterpret_cast<int4 *>(meta + L.tile_desc + 4 * (int64_t)idx) =
                 make_int4(s, r0, rows | (contiguous << 15) | (e.rank << 16), __float_as_int(e.scale));
-            // private list of 16-row pieces (all earlier tiles of the segment are full)
+            // private unit records: the tile's pieces of at most 16 rows (all earlier tiles of the
+            // segment are full, so they have ppt pieces each)
             for (int32_t i = 0; i < (rows + 15) / 16; ++i)
-                meta[L.tile_piece + piece0[s] + k * ppt + i] = (idx << 4) | i;
+                *reinterpret_cast<int4 *>(meta + L.unit_desc + 4 * (int64_t)(piece0[s] + k * ppt + i)) =
+                    make_int4(s, r0 + 16 * i,
+                              min(16, rows - 16 * i) | (rows << 8) | (contiguous << 16) | (e.rank << 17),
+                              __float_as_int(e.scale));
         }
     }
 

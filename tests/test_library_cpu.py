@@ -83,8 +83,8 @@ def test_segments_bytes_matches_documented_layout():
     public_words = words
     words = (words + 3) // 4 * 4 + 4 * cap_tile          # library-private tile records
     desc_end = words
-    words += cap_tile * tile_m                           # library-private per-tile row ids
-    words += cap_tile * ((tile_m + 15) // 16)            # library-private list of 16-row pieces
+    cap_unit = cap_tile * ((tile_m + 15) // 16)          # 16-row pieces of all tiles
+    words += 4 * cap_unit + 16 * cap_unit                # library-private unit records and row ids
     assert lb.segments_bytes(T, N, tile_m) == 4 * words
     assert lb.segments_bytes(0, N, tile_m) == 4 * 20
     with pytest.raises(lb.LoraError):
