@@ -45,7 +45,7 @@ struct FusedMaps {
     CUtensorMap a[8], b[8];
 };
 #ifndef LORA_FUSED_MIN_BLOCKS
-#define LORA_FUSED_MIN_BLOCKS 5   // resident blocks per SM the register budget is held to
+#define LORA_FUSED_MIN_BLOCKS 6   // resident blocks per SM the register budget is held to
 #endif
 
 // ---------------------------------------------------------------------------------------------
@@ -253,22 +253,31 @@ struct Ctx {
     bool ok;                   // no wait has expired
 };
 
-// Warp 0: request jobs until the ring is full.  Jobs of the unit after the current one may be
-// requested (their record is already in the ring); anything further ahead waits.
-__device__ __forceinline__ void issue_jobs(const ApplyParams &P, const FusedMaps &M, Ctx &cx, int lane) {
+// Position in the block's job stream -> the job's unit and row ids.  Moves (it_i, it_j) past
+// units without jobs.  False when the stream has no further job that may be requested yet: jobs of
+// the unit after the current one may be (their record is in the ring), anything further waits.
+__device__ __forceinline__ bool peek_job(const ApplyParams &P, const Ctx &cx, int32_t &it_i, int32_t &it_j,
+                                         Unit &un, const int32_t *&rowidx) {
+    for (;;) {
+        if (it_i > cx.ci + 1 || cx.cid + it_i * cx.G >= cx.n_units) return false;
+        const unsigned char *e = cx.smem + SM_RING + (it_i % UNIT_RING) * RING_ENTRY;
+        un = decode_unit(P, *reinterpret_cast<const int4 *>(e), cx.a_hi - cx.a_lo, cx.b_hi - cx.b_lo);
+        rowidx = reinterpret_cast<const int32_t *>(e + 16);
+        if (un.run && it_j < un.na + un.nb) return true;
+        ++it_i;
+        it_j = 0;
+    }
+}
+
+// Warp 0: request jobs until the ring is full.
+// mode 0: whole jobs; 1: only the weight tiles (and the byte count of the whole job); 2: only the
+// token rows of jobs whose weight tiles were requested in mode 1 (same walk, from the same state).
+__device__ __forceinline__ void issue_jobs(const ApplyParams &P, const FusedMaps &M, Ctx &cx, int lane,
+                                           int mode = 0) {
     const int32_t S = P.n_stages;
-    while (cx.pq - cx.cq < S) {
-        Unit un;
-        const int32_t *rowidx;
-        for (;;) {
-            if (cx.pi > cx.ci + 1 || cx.cid + cx.pi * cx.G >= cx.n_units) return;
-            const unsigned char *e = cx.smem + SM_RING + (cx.pi % UNIT_RING) * RING_ENTRY;
-            un = decode_unit(P, *reinterpret_cast<const int4 *>(e), cx.a_hi - cx.a_lo, cx.b_hi - cx.b_lo);
-            rowidx = reinterpret_cast<const int32_t *>(e + 16);
-            if (un.run && cx.pj < un.na + un.nb) break;
-            ++cx.pi;
-            cx.pj = 0;
-        }
+    Unit un;
+    const int32_t *rowidx;
+    while (cx.pq - cx.cq < S && peek_job(P, cx, cx.pi, cx.pj, un, rowidx)) {
         const int st = cx.pq % S;
         unsigned char *ws = cx.smem + P.off_stage + st * P.stage_bytes;
         const bool shrink = cx.pj < un.na;
@@ -280,14 +289,14 @@ __device__ __forceinline__ void issue_jobs(const ApplyParams &P, const FusedMaps
         const __nv_bfloat16 *tok = (shrink ? P.x : P.yb) + col0;
         const int64_t tld = shrink ? P.ldx : P.ldyb;
         __nv_bfloat16 *ts = reinterpret_cast<__nv_bfloat16 *>(ws + W_BYTES);
-        if (lane == 0) {
+        if (lane == 0 && mode != 2) {
             // the tile load always delivers its whole box: rb rows of CW columns
             mbar_expect_tx(&cx.full[st], (uint32_t)un.rb * (uint32_t)un.CW * 2u +
                                              (uint32_t)un.rows * (uint32_t)ncols * 2u);
             tma_load_4d(ws, map, 0, 0, col0 >> 6, un.slot, &cx.full[st]);
         }
         __syncwarp();
-        if (lane < un.rows)
+        if (lane < un.rows && mode != 1)
             bulk_g2s(ts + lane * pitch, tok + (int64_t)rowidx[lane] * tld, (uint32_t)ncols * 2u,
                      &cx.full[st]);
         ++cx.pj;
@@ -337,9 +346,22 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
     const uint32_t blk_bytes = (uint32_t)un.rb * 128u;
 
     // ---- shrink: warp w takes columns [w*KW, (w+1)*KW) of every chunk (split-K) ------------------
-    float acc[NT_S][4];
+    // Partial sums live in registers across the unit's jobs, except for the widest rank bucket:
+    // there a warp has one MMA step per job, and adding each job's result into the warp's slot of
+    // `part` keeps 28 registers free (each thread updates only elements it owns).
+    constexpr bool PARK = NT_S > 4;
+    float acc[PARK ? 1 : NT_S][4];
+    float *mypart = part + (warp * mrows + g) * RP + 2 * t;
+    if (PARK) {
 #pragma unroll
-    for (int nt = 0; nt < NT_S; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.0f;
+        for (int nt = 0; nt < NT_S; ++nt) {
+            *reinterpret_cast<float2 *>(mypart + nt * 8) = make_float2(0.0f, 0.0f);
+            if (hi_rows) *reinterpret_cast<float2 *>(mypart + nt * 8 + 8 * RP) = make_float2(0.0f, 0.0f);
+        }
+    } else {
+#pragma unroll
+        for (int nt = 0; nt < (PARK ? 1 : NT_S); ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.0f;
+    }
     for (int32_t c = 0; c < un.na; ++c) {
         const unsigned char *As = acquire_job(P, cx);   // tile of A_i, then [mrows][PW] rows of x
         const __nv_bfloat16 *X = reinterpret_cast<const __nv_bfloat16 *>(As + W_BYTES);
@@ -357,9 +379,22 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
                 const unsigned char *ab = As + (uint32_t)(kk >> 6) * blk_bytes + g * 128 + 4 * t;
                 const uint32_t ch = (uint32_t)(kk & 63) >> 3;   // even
 #pragma unroll
-                for (int nt = 0; nt < NT_S; ++nt)
-                    mma16816(acc[nt], a, lds32b(ab + nt * 1024 + ((ch ^ (uint32_t)g) << 4)),
-                             full ? lds32b(ab + nt * 1024 + (((ch + 1) ^ (uint32_t)g) << 4)) : 0u);
+                for (int nt = 0; nt < NT_S; ++nt) {
+                    const uint32_t b0 = lds32b(ab + nt * 1024 + ((ch ^ (uint32_t)g) << 4));
+                    const uint32_t b1 = full ? lds32b(ab + nt * 1024 + (((ch + 1) ^ (uint32_t)g) << 4)) : 0u;
+                    if (PARK) {
+                        float d[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                        mma16816(d, a, b0, b1);
+                        float2 *p0 = reinterpret_cast<float2 *>(mypart + nt * 8);
+                        *p0 = make_float2(p0->x + d[0], p0->y + d[1]);
+                        if (hi_rows) {
+                            float2 *p1 = reinterpret_cast<float2 *>(mypart + nt * 8 + 8 * RP);
+                            *p1 = make_float2(p1->x + d[2], p1->y + d[3]);
+                        }
+                    } else {
+                        mma16816(acc[PARK ? 0 : nt], a, b0, b1);
+                    }
+                }
             }
         }
         release_job(P, M, cx, warp, lane);
@@ -369,11 +404,12 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
         cluster_wait();
         cx.pending_wait = false;
     }
+    if (!PARK) {
 #pragma unroll
-    for (int nt = 0; nt < NT_S; ++nt) {
-        float *p0 = part + (warp * mrows + g) * RP + nt * 8 + 2 * t;
-        *reinterpret_cast<float2 *>(p0) = make_float2(acc[nt][0], acc[nt][1]);
-        if (hi_rows) *reinterpret_cast<float2 *>(p0 + 8 * RP) = make_float2(acc[nt][2], acc[nt][3]);
+        for (int nt = 0; nt < (PARK ? 1 : NT_S); ++nt) {
+            *reinterpret_cast<float2 *>(mypart + nt * 8) = make_float2(acc[nt][0], acc[nt][1]);
+            if (hi_rows) *reinterpret_cast<float2 *>(mypart + nt * 8 + 8 * RP) = make_float2(acc[nt][2], acc[nt][3]);
+        }
     }
     __syncthreads();
     // block partial: the four warps' sums in warp order
@@ -416,10 +452,15 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
         const __nv_bfloat16 *Ys = reinterpret_cast<const __nv_bfloat16 *>(Bs + W_BYTES);
         const int32_t col0 = cx.b_lo + c * CW, ncols = min(CW, cx.b_hi - col0);
         const int base = warp * NW;
-        if (base < ncols) {
-            float ex[NT_E][4];
+        // column tiles in groups of at most four: 16 accumulator registers at a time
+        constexpr int NG = NT_E < 4 ? NT_E : 4;
 #pragma unroll
-            for (int j = 0; j < NT_E; ++j) ex[j][0] = ex[j][1] = ex[j][2] = ex[j][3] = 0.0f;
+        for (int j0 = 0; j0 < NT_E; j0 += NG) {
+            const int gbase = base + j0 * 8;
+            if (gbase >= ncols) break;
+            float ex[NG][4];
+#pragma unroll
+            for (int j = 0; j < NG; ++j) ex[j][0] = ex[j][1] = ex[j][2] = ex[j][3] = 0.0f;
             const __nv_bfloat16 *vh = Vh + g * PV + 2 * t;
             const __nv_bfloat16 *vl = Vl + g * PV + 2 * t;
             for (int ks = 0; ks < rank16; ks += 16) {
@@ -433,10 +474,10 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
                 al[2] = lds32(vl + ks + 8);
                 al[3] = hi_rows ? lds32(vl + 8 * PV + ks + 8) : 0u;
 #pragma unroll
-                for (int np = 0; np < NT_E / 2; ++np) {
+                for (int np = 0; np < NG / 2; ++np) {
                     // matrices: (k 0..7, tile 2np), (k 8..15, tile 2np), (k 0..7, 2np+1), (k 8..15, 2np+1)
                     const int mi = lane >> 3;
-                    const int col = base + (np * 2 + (mi >> 1)) * 8;
+                    const int col = gbase + (np * 2 + (mi >> 1)) * 8;
                     const unsigned char *bp = Bs + (uint32_t)(col >> 6) * blk_bytes +
                                               (ks + (mi & 1) * 8 + (lane & 7)) * 128 +
                                               ((((uint32_t)(col & 63) >> 3) ^ (uint32_t)(lane & 7)) << 4);
@@ -454,11 +495,11 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
             for (int h = 0; h < H; ++h) {
                 const int32_t m = g + 8 * h;
                 if (m < rows && cx.ok) {
-                    __nv_bfloat16 *yrow = P.y + (int64_t)rowidx[m] * P.ldy + col0 + base + 2 * t;
-                    const __nv_bfloat16 *ybrow = Ys + m * PW + base + 2 * t;
+                    __nv_bfloat16 *yrow = P.y + (int64_t)rowidx[m] * P.ldy + col0 + gbase + 2 * t;
+                    const __nv_bfloat16 *ybrow = Ys + m * PW + gbase + 2 * t;
 #pragma unroll
-                    for (int j = 0; j < NT_E; ++j) {
-                        if (base + j * 8 < ncols) {
+                    for (int j = 0; j < NG; ++j) {
+                        if (gbase + j * 8 < ncols) {
                             const uint32_t w = lds32(ybrow + j * 8);
                             const float y0 = fmaf(s, ex[j][2 * h], __uint_as_float(w << 16));
                             const float y1 = fmaf(s, ex[j][2 * h + 1], __uint_as_float(w & 0xffff0000u));
@@ -491,21 +532,11 @@ fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
         return;
     }
 
-    // set-up that touches no global memory: barriers, and zeros in every stage (rows above a
-    // unit's rank are never copied, and what they hold is multiplied by zeros of v)
+    // barriers; the next lines touch no memory another kernel writes
     if (tid == 0) {
         for (int s = 0; s < P.n_stages; ++s) mbar_init(&cx.full[s], 1);
         fence_mbar_init();
     }
-    for (int i = tid; i < P.n_stages * P.stage_bytes / 16; i += FT)
-        reinterpret_cast<uint4 *>(smem + P.off_stage)[i] = make_uint4(0, 0, 0, 0);
-    fence_proxy_async();   // the stages are written by bulk copies from here on
-    // the next kernel on the stream may be scheduled from here on, and this one waits for
-    // everything queued before it
-    griddep_launch_dependents();
-    __syncthreads();
-    griddep_wait();
-
     // this block's column slices (multiples of 64 columns: tile loads address whole column blocks)
     {
         const int32_t cs64 = (int32_t)cx.csize * 64;
@@ -515,14 +546,24 @@ fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
         cx.b_lo = min((int32_t)cx.crank * Wb, P.tv.d_out);
         cx.b_hi = min(cx.b_lo + Wb, P.tv.d_out);
     }
-    // the number of units and the records of this cluster's first two units, side by side
+    // Under programmatic dependent launch this kernel may start while the one before it on the
+    // stream is still running.  Activations are only touched after griddep_wait().  The unit
+    // records and the pool were complete before that kernel started when P.early is set (the host
+    // sets it only then), so they are read, and the first weight tiles requested, ahead of the wait.
+    if (!P.early) griddep_wait();
     {
+        // the number of units and the records of this cluster's first two units, side by side
         UnitRegs m0, m1;
         if (warp == 3) {
             m0 = fetch_unit(P, cx.cid, P.units, lane);
             m1 = fetch_unit(P, cx.cid + cx.G, P.units, lane);
         }
         cx.n_units = P.meta ? ldg_int(P.meta + H_NPIECE) : P.T;
+        // meanwhile: zeros in every stage (rows above a unit's rank are never copied, and what
+        // they hold is multiplied by zeros of v, so it has to be finite)
+        for (int i = tid; i < P.n_stages * P.stage_bytes / 16; i += FT)
+            reinterpret_cast<uint4 *>(smem + P.off_stage)[i] = make_uint4(0, 0, 0, 0);
+        fence_proxy_async();   // the stages are written by bulk copies from here on
         if (cx.n_units > P.units) cx.n_units = P.units;
         if (warp == 3) {
             store_unit(smem, 0, m0, cx.cid < cx.n_units, lane);
@@ -534,6 +575,17 @@ fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
     cx.cq = cx.pq = cx.pi = cx.pj = 0;
     cx.pending_wait = false;
     cx.ok = true;
+    if (P.early) {
+        if (warp == 0) issue_jobs(P, M, cx, lane, 1);
+        griddep_wait();
+        if (warp == 0) {
+            cx.pi = cx.pj = cx.pq = 0;
+            issue_jobs(P, M, cx, lane, 2);
+        }
+    }
+    // the next kernel on the stream may be scheduled from here on: everything older than this
+    // kernel is complete
+    griddep_launch_dependents();
 
     for (;; ++cx.ci) {
         const int32_t u = cx.cid + cx.ci * cx.G;
@@ -656,7 +708,7 @@ static lora_status_t launch_h(lora_pool_t *pool, ApplyParams P, int32_t C, const
     // a stage: the weight tile, then the token rows at the widest chunk (rank bucket 16)
     const int32_t stage = (W_BYTES + mrows * (256 + 8) * 2 + 1023) & ~1023;
     int32_t S = pool->tuning[5];
-    if (S < 2 || S > MAX_STAGES) S = 3;
+    if (S < 2 || S > MAX_STAGES) S = 2;   // two stages and more resident blocks beat deeper rings
     int32_t o = SM_HEADER;
     P.off_part = o;   o += 4 * mrows * RPmax * 4;
     P.off_vpart = o;  o += mrows * RPmax * 4;
@@ -685,7 +737,12 @@ static lora_status_t launch_h(lora_pool_t *pool, ApplyParams P, int32_t C, const
     at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
-    const unsigned n_attrs = pool->tuning[2] == 1 ? 2 : 1;   // tuning key 2 = 1: programmatic dependent launch
+    // Programmatic dependent launch (tuning key 2: 0 = when allowed, 2 = never).  Allowed for
+    // grouped batches whose table has already been read by an earlier apply: that apply was fully
+    // ordered behind the build, so the table is complete before this kernel can start.
+    const bool fresh = P.meta ? pool->take_fresh(P.meta) : true;
+    P.early = (P.meta && !fresh && pool->tuning[2] != 2) ? 1 : 0;
+    const unsigned n_attrs = P.early ? 2 : 1;
 
     // Grid: no more clusters than can be resident at once (each loops over its units), so no
     // cluster of an over-sized grid waits for a slot only to find that its unit does not exist.

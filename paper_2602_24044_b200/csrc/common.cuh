@@ -146,16 +146,17 @@ struct lora_pool {
     struct MetaRecord {
         const void *ptr;
         int32_t T, tile_m, long_min;
+        bool fresh;   // built, and no apply has been queued behind the build yet
     };
     std::vector<MetaRecord> metas;
     void remember_meta(const void *ptr, int32_t T, int32_t tile_m, int32_t long_min) {
         for (MetaRecord &m : metas)
             if (m.ptr == ptr) {
-                m.T = T; m.tile_m = tile_m; m.long_min = long_min;
+                m.T = T; m.tile_m = tile_m; m.long_min = long_min; m.fresh = true;
                 return;
             }
         if (metas.size() >= 256) metas.erase(metas.begin());
-        metas.push_back({ptr, T, tile_m, long_min});
+        metas.push_back({ptr, T, tile_m, long_min, true});
     }
     bool find_meta(const void *ptr, int32_t T, int32_t *tile_m) const {
         for (const MetaRecord &m : metas)
@@ -164,6 +165,18 @@ struct lora_pool {
                 return true;
             }
         return false;
+    }
+
+    // True once for a table after each build: the first kernel that reads the table must be
+    // fully ordered behind the build; later ones may read it before their predecessor has finished.
+    bool take_fresh(const void *ptr) {
+        for (MetaRecord &m : metas)
+            if (m.ptr == ptr) {
+                const bool f = m.fresh;
+                m.fresh = false;
+                return f;
+            }
+        return true;
     }
 
     lora::PoolView view() const {
