@@ -381,8 +381,8 @@ def main():
     # swap-in on the side stream while steps run (config 4: 16 misses per step)
     swap = None
     if cfg == 4 and rank == 0:
-        blobs = s.host_adapter(0, lb.A_RANK_MAJOR)
-        adapter_bytes = sum(int(t.numel()) * 2 for t in blobs[0] + blobs[1])
+        blobs = s.host_adapter_packed(0)      # one pinned buffer per adapter: a single DMA per miss
+        adapter_bytes = int(blobs[0][0].numel()) * 2
         steps_sw = 5
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         l0e, l1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -392,7 +392,7 @@ def main():
         for i in range(steps_sw):
             for v in wl.swap_victims:
                 lb.pool_load_slot(s.pool, v, int(wl.ranks[v]), float(wl.scales[v]), blobs[0], blobs[1],
-                                  lb.A_RANK_MAJOR, s.load, None, True)
+                                  lb.PACKED, s.load, None, True)
             run_steps(1, g_step, step)
         ev1.record(s.compute)
         l1e.record(s.load)

@@ -91,14 +91,18 @@ lora_status_t lora_pool_create(const lora_pool_desc_t *desc, lora_pool_t **out);
 lora_status_t lora_pool_destroy(lora_pool_t *pool);
 
 enum { LORA_A_DIN_MAJOR = 0,   /* A given as [d_in, rank] row-major (the formula's orientation) */
-       LORA_A_RANK_MAJOR = 1   /* A given as [rank, d_in] row-major (already in slot layout)    */ };
+       LORA_A_RANK_MAJOR = 1,  /* A given as [rank, d_in] row-major (already in slot layout)    */
+       LORA_PACKED = 2         /* A[0] is ONE pinned buffer (16-byte aligned) holding, for every
+                                  target in order, A as [rank, d_in] then B as [rank, d_out]; the
+                                  other pointers are ignored.  With rank == r_max this is the slot's
+                                  own layout and the swap-in is a single DMA. */ };
 
 typedef struct {
     int32_t rank;            /* 1 .. r_max */
     float scale;             /* s_i */
     const void *const *A;    /* host, [num_targets] pointers to pinned bf16 matrices, see a_layout */
     const void *const *B;    /* host, [num_targets] pointers to pinned bf16 [rank, d_out] row-major */
-    int32_t a_layout;        /* LORA_A_DIN_MAJOR or LORA_A_RANK_MAJOR */
+    int32_t a_layout;        /* LORA_A_DIN_MAJOR, LORA_A_RANK_MAJOR or LORA_PACKED */
     int32_t trust_pinned;    /* non-zero: skip the per-pointer pinned-memory check */
 } lora_adapter_host_t;
 

@@ -18,6 +18,7 @@ from . import build as _build
 LORA_OK = 0
 A_DIN_MAJOR = 0
 A_RANK_MAJOR = 1
+PACKED = 2
 META_HEADER_WORDS = 16
 
 EXPORTS = [

@@ -10,14 +10,14 @@
 // (TMA, 128-byte swizzle, the matrix viewed as blocks of 64 columns), plus the unit's rows of x (or
 // y_base), one bulk copy per row, into one stage of a small ring of shared-memory buffers
 // (mbarrier-signalled).  Few large copies matter: every bulk copy costs the issuing thread and the
-// copy engine a fixed time, and a copy per weight row made that time the bottleneck.  Warp 0 keeps the ring full: whenever a stage has been consumed it
-// requests the next job of the stream, which may belong to the next unit, so the memory latency of
+// copy engine a fixed time, and a copy per weight row made that time the bottleneck.  Warp 0 keeps
+// the ring full: whenever a stage has been consumed it requests the next job of the stream, which may belong to the next unit, so the memory latency of
 // a unit hides behind the arithmetic of the one before.  The chunk width shrinks as the rank
 // grows (256 / 128 / 64 columns for ranks <= 16 / 32 / 64), so a stage is the same size for
 // every rank and one launch serves all of them.
 //
-//   shrink  partial v over the block's d_in slice, split-K over the four warps, bf16 tensor-core
-//           MMA (m16n8k16) with fp32 accumulation carried across chunks in registers;
+//   shrink  partial v over the block's d_in slice, the four warps splitting rank tiles and columns,
+//           bf16 tensor-core MMA (m16n8k16) with fp32 accumulation carried across chunks in registers;
 //   exchange the block partials are summed through distributed shared memory in block order,
 //           identically in every block (no global workspace, no float atomics);
 //   expand  over the block's d_out slice on the tensor cores, v carried as the sum of two bf16
@@ -325,15 +325,17 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
     constexpr int CW = 4096 / RP;      // columns per job
     constexpr int PW = CW + 8;         // row pitch of the token rows: +16 B against bank conflicts
     constexpr int PV = RP + 8;         // pitch of the bf16 copies of v
-    constexpr int NT_S = RP / 8;       // rank tiles of 8 in the shrink MMA
-    constexpr int KW = CW / 4;         // shrink: columns per warp and job (split-K)
+    // shrink: the four warps split the rank tiles WN ways and the chunk's columns WK ways, so that
+    // every warp owns two rank tiles of 8 and 64 columns of every job, whatever the bucket
+    constexpr int WN = RP / 16, WK = 4 / WN;
+    constexpr int KW = CW / WK;        // = 64 columns per warp and job
     constexpr int NW = CW / 4;         // expand: columns per warp and job
     constexpr int NT_E = NW / 8;       // expand: column tiles of 8 per warp
     constexpr int mrows = 8 * H;
     constexpr bool hi_rows = H == 2;
 
     unsigned char *smem = cx.smem;
-    float *part = reinterpret_cast<float *>(smem + P.off_part);     // [4 warps][mrows][RP]
+    float *part = reinterpret_cast<float *>(smem + P.off_part);     // [WK][mrows][RP] = mrows x 64 floats
     float *vpart = reinterpret_cast<float *>(smem + P.off_vpart);   // [mrows][RP], read by the peers
     __nv_bfloat16 *Vh = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_vh);   // [mrows][PV]
     __nv_bfloat16 *Vl = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_vl);
@@ -345,30 +347,18 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
     // chunks of a row exchanged by the row number's low three bits (128-byte swizzle).
     const uint32_t blk_bytes = (uint32_t)un.rb * 128u;
 
-    // ---- shrink: warp w takes columns [w*KW, (w+1)*KW) of every chunk (split-K) ------------------
-    // Partial sums live in registers across the unit's jobs, except for the widest rank bucket:
-    // there a warp has one MMA step per job, and adding each job's result into the warp's slot of
-    // `part` keeps 28 registers free (each thread updates only elements it owns).
-    constexpr bool PARK = NT_S > 4;
-    float acc[PARK ? 1 : NT_S][4];
-    float *mypart = part + (warp * mrows + g) * RP + 2 * t;
-    if (PARK) {
+    // ---- shrink: warp (wk, wn) takes columns [wk*KW, (wk+1)*KW) of every chunk and rank tiles 2wn, 2wn+1
+    const int wk = warp % WK, wn = warp / WK;
+    float acc[2][4];
 #pragma unroll
-        for (int nt = 0; nt < NT_S; ++nt) {
-            *reinterpret_cast<float2 *>(mypart + nt * 8) = make_float2(0.0f, 0.0f);
-            if (hi_rows) *reinterpret_cast<float2 *>(mypart + nt * 8 + 8 * RP) = make_float2(0.0f, 0.0f);
-        }
-    } else {
-#pragma unroll
-        for (int nt = 0; nt < (PARK ? 1 : NT_S); ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.0f;
-    }
+    for (int i = 0; i < 2; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.0f;
     for (int32_t c = 0; c < un.na; ++c) {
         const unsigned char *As = acquire_job(P, cx);   // tile of A_i, then [mrows][PW] rows of x
         const __nv_bfloat16 *X = reinterpret_cast<const __nv_bfloat16 *>(As + W_BYTES);
         const int32_t ncols = min(CW, cx.a_hi - (cx.a_lo + c * CW));
 #pragma unroll
         for (int ks = 0; ks < KW; ks += 16) {
-            const int kk = warp * KW + ks;
+            const int kk = wk * KW + ks;
             if (kk < ncols) {
                 const bool full = ncols - kk >= 16;   // else only 8 columns are left
                 uint32_t a[4];
@@ -379,21 +369,10 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
                 const unsigned char *ab = As + (uint32_t)(kk >> 6) * blk_bytes + g * 128 + 4 * t;
                 const uint32_t ch = (uint32_t)(kk & 63) >> 3;   // even
 #pragma unroll
-                for (int nt = 0; nt < NT_S; ++nt) {
-                    const uint32_t b0 = lds32b(ab + nt * 1024 + ((ch ^ (uint32_t)g) << 4));
-                    const uint32_t b1 = full ? lds32b(ab + nt * 1024 + (((ch + 1) ^ (uint32_t)g) << 4)) : 0u;
-                    if (PARK) {
-                        float d[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                        mma16816(d, a, b0, b1);
-                        float2 *p0 = reinterpret_cast<float2 *>(mypart + nt * 8);
-                        *p0 = make_float2(p0->x + d[0], p0->y + d[1]);
-                        if (hi_rows) {
-                            float2 *p1 = reinterpret_cast<float2 *>(mypart + nt * 8 + 8 * RP);
-                            *p1 = make_float2(p1->x + d[2], p1->y + d[3]);
-                        }
-                    } else {
-                        mma16816(acc[PARK ? 0 : nt], a, b0, b1);
-                    }
+                for (int i = 0; i < 2; ++i) {
+                    const int nt = wn * 2 + i;
+                    mma16816(acc[i], a, lds32b(ab + nt * 1024 + ((ch ^ (uint32_t)g) << 4)),
+                             full ? lds32b(ab + nt * 1024 + (((ch + 1) ^ (uint32_t)g) << 4)) : 0u);
                 }
             }
         }
@@ -404,19 +383,22 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
         cluster_wait();
         cx.pending_wait = false;
     }
-    if (!PARK) {
 #pragma unroll
-        for (int nt = 0; nt < (PARK ? 1 : NT_S); ++nt) {
-            *reinterpret_cast<float2 *>(mypart + nt * 8) = make_float2(acc[nt][0], acc[nt][1]);
-            if (hi_rows) *reinterpret_cast<float2 *>(mypart + nt * 8 + 8 * RP) = make_float2(acc[nt][2], acc[nt][3]);
-        }
+    for (int i = 0; i < 2; ++i) {
+        float *p0 = part + (wk * mrows + g) * RP + (wn * 2 + i) * 8 + 2 * t;
+        *reinterpret_cast<float2 *>(p0) = make_float2(acc[i][0], acc[i][1]);
+        if (hi_rows) *reinterpret_cast<float2 *>(p0 + 8 * RP) = make_float2(acc[i][2], acc[i][3]);
     }
     __syncthreads();
-    // block partial: the four warps' sums in warp order
+    // block partial: the column splits' sums in order
     for (int i = tid; i < mrows * RP; i += FT) {
         const int r = i / RP;
-        if (r < rows)
-            vpart[i] = ((part[i] + part[mrows * RP + i]) + part[2 * mrows * RP + i]) + part[3 * mrows * RP + i];
+        if (r < rows) {
+            float v = part[i];
+#pragma unroll
+            for (int w = 1; w < WK; ++w) v += part[w * mrows * RP + i];
+            vpart[i] = v;
+        }
     }
     // ---- exchange: every block sums all blocks' partials in block order -------------------------
     cluster_arrive();
@@ -710,7 +692,7 @@ static lora_status_t launch_h(lora_pool_t *pool, ApplyParams P, int32_t C, const
     int32_t S = pool->tuning[5];
     if (S < 2 || S > MAX_STAGES) S = 2;   // two stages and more resident blocks beat deeper rings
     int32_t o = SM_HEADER;
-    P.off_part = o;   o += 4 * mrows * RPmax * 4;
+    P.off_part = o;   o += mrows * 64 * 4;
     P.off_vpart = o;  o += mrows * RPmax * 4;
     P.off_vh = o;     o += mrows * (RPmax + 8) * 2;
     P.off_vl = o;     o += mrows * (RPmax + 8) * 2;

@@ -179,17 +179,37 @@ lora_status_t lora_pool_load_slot(lora_pool_t *pool, int32_t slot, const lora_ad
     if (!pool || !ad || !ad->A || !ad->B) return LORA_ERR_INVALID_ARG;
     if (slot < 0 || slot >= pool->num_slots) return LORA_ERR_SLOT_RANGE;
     if (ad->rank < 1 || ad->rank > pool->r_max) return LORA_ERR_RANK;
-    if (ad->a_layout != LORA_A_DIN_MAJOR && ad->a_layout != LORA_A_RANK_MAJOR)
+    if (ad->a_layout != LORA_A_DIN_MAJOR && ad->a_layout != LORA_A_RANK_MAJOR &&
+        ad->a_layout != LORA_PACKED)
         return LORA_ERR_INVALID_ARG;
-    for (int32_t t = 0; t < pool->num_targets; ++t) {
-        if (!ad->A[t] || !ad->B[t]) return LORA_ERR_INVALID_ARG;
-        if (((uintptr_t)ad->A[t] | (uintptr_t)ad->B[t]) & 1) return LORA_ERR_INVALID_ARG;
+    const bool packed = ad->a_layout == LORA_PACKED;
+    // packed: A[0] is one buffer with every target's A [rank, d_in] and B [rank, d_out] in order
+    std::vector<const char *> srcA(pool->num_targets), srcB(pool->num_targets);
+    if (packed) {
+        if (!ad->A[0] || ((uintptr_t)ad->A[0] & 15)) return LORA_ERR_INVALID_ARG;
+        const char *p = (const char *)ad->A[0];
+        for (int32_t t = 0; t < pool->num_targets; ++t) {
+            srcA[t] = p;  p += (size_t)ad->rank * pool->targets[t].d_in * 2;
+            srcB[t] = p;  p += (size_t)ad->rank * pool->targets[t].d_out * 2;
+        }
+    } else {
+        for (int32_t t = 0; t < pool->num_targets; ++t) {
+            if (!ad->A[t] || !ad->B[t]) return LORA_ERR_INVALID_ARG;
+            if (((uintptr_t)ad->A[t] | (uintptr_t)ad->B[t]) & 1) return LORA_ERR_INVALID_ARG;
+            srcA[t] = (const char *)ad->A[t];
+            srcB[t] = (const char *)ad->B[t];
+        }
     }
     DeviceGuard guard(pool->device);
     if (!guard.ok) return cuda_fail(cudaErrorInvalidDevice);
-    if (!ad->trust_pinned)
-        for (int32_t t = 0; t < pool->num_targets; ++t)
-            if (!is_pinned(ad->A[t]) || !is_pinned(ad->B[t])) return LORA_ERR_NOT_PINNED;
+    if (!ad->trust_pinned) {
+        if (packed) {
+            if (!is_pinned(srcA[0]) || !is_pinned(srcB[pool->num_targets - 1])) return LORA_ERR_NOT_PINNED;
+        } else {
+            for (int32_t t = 0; t < pool->num_targets; ++t)
+                if (!is_pinned(ad->A[t]) || !is_pinned(ad->B[t])) return LORA_ERR_NOT_PINNED;
+        }
+    }
 
     cudaStream_t ls = (cudaStream_t)load_stream, cs = (cudaStream_t)compute_stream;
     if (!pool->ready[slot])
@@ -203,17 +223,23 @@ lora_status_t lora_pool_load_slot(lora_pool_t *pool, int32_t slot, const lora_ad
     set_slot_kernel<<<1, 32, 0, ls>>>(pool->table_dev, slot, 0, 0.0f, 0);
     if ((s = count_launch()) != LORA_OK) return s;
 
-    // One DMA per matrix.  Neighbouring host matrices are not merged into one copy: two pinned
-    // allocations can be adjacent in the address space, and a copy must not span both.
+    // One DMA per matrix.  Neighbouring host matrices given as separate pointers are not merged
+    // into one copy: two pinned allocations can be adjacent in the address space, and a copy must
+    // not span both.  A caller that holds the adapter in one buffer says so with LORA_PACKED.
     std::vector<CopyJob> jobs;
     auto push = [&jobs](void *dst, const void *src, size_t bytes) {
         jobs.push_back({(char *)dst, (const char *)src, bytes});
     };
-    for (int32_t t = 0; t < pool->num_targets; ++t) {
-        const TargetView &tv = pool->target_views[t];
-        if (ad->a_layout == LORA_A_RANK_MAJOR)
-            push(slot_base + tv.off_a, ad->A[t], (size_t)r * tv.d_in * 2);
-        push(slot_base + tv.off_b, ad->B[t], (size_t)r * tv.d_out * 2);
+    if (packed && r == r8) {
+        // a full-rank packed adapter has exactly the slot's layout: one DMA for the whole adapter
+        push(slot_base, srcA[0], (size_t)pool->slot_stride * 2);
+    } else {
+        for (int32_t t = 0; t < pool->num_targets; ++t) {
+            const TargetView &tv = pool->target_views[t];
+            if (ad->a_layout != LORA_A_DIN_MAJOR)
+                push(slot_base + tv.off_a, srcA[t], (size_t)r * tv.d_in * 2);
+            push(slot_base + tv.off_b, srcB[t], (size_t)r * tv.d_out * 2);
+        }
     }
     for (const CopyJob &j : jobs)
         LORA_CUDA_TRY(cudaMemcpyAsync(j.dst, j.src, j.bytes, cudaMemcpyHostToDevice, ls));
@@ -222,7 +248,7 @@ lora_status_t lora_pool_load_slot(lora_pool_t *pool, int32_t slot, const lora_ad
         const TargetView &tv = pool->target_views[t];
         __nv_bfloat16 *dA = slot_base + tv.off_a, *dB = slot_base + tv.off_b;
         if (ad->a_layout == LORA_A_DIN_MAJOR) {
-            LORA_CUDA_TRY(cudaMemcpyAsync(pool->staging_dev, ad->A[t], (size_t)r * tv.d_in * 2,
+            LORA_CUDA_TRY(cudaMemcpyAsync(pool->staging_dev, srcA[t], (size_t)r * tv.d_in * 2,
                                           cudaMemcpyHostToDevice, ls));
             transpose_a_kernel<<<(tv.d_in + 255) / 256, 256, 0, ls>>>(pool->staging_dev, dA,
                                                                       tv.d_in, r, r8);

@@ -80,11 +80,25 @@ class Session:
             B.append(bf16_tensor(b, pin=True))
         return A, B
 
+    def host_adapter_packed(self, slot: int):
+        """One pinned buffer with every target's A [rank, d_in] and B [rank, d_out] in order."""
+        parts = []
+        for t in self.target_ids:
+            a, b = self.wl.adapter_weights(slot, t)
+            parts += [np.ascontiguousarray(a.T).ravel(), np.ascontiguousarray(b).ravel()]
+        buf = bf16_tensor(np.concatenate(parts), pin=True)
+        return [buf] * len(self.target_ids), [buf] * len(self.target_ids)
+
     def load_slot(self, slot: int, a_layout: int = lb.A_DIN_MAJOR, src_slot: Optional[int] = None,
                   rank: Optional[int] = None, scale: Optional[float] = None, blobs=None):
         """Queue a swap-in of the workload's adapter `src_slot` (default: `slot`) into `slot`."""
         src = slot if src_slot is None else src_slot
-        A, B = blobs if blobs is not None else self.host_adapter(src, a_layout)
+        if blobs is not None:
+            A, B = blobs
+        elif a_layout == lb.PACKED:
+            A, B = self.host_adapter_packed(src)
+        else:
+            A, B = self.host_adapter(src, a_layout)
         self._pinned += A + B
         lb.pool_load_slot(self.pool, slot, int(self.wl.ranks[src]) if rank is None else rank,
                           float(self.wl.scales[src]) if scale is None else scale, A, B, a_layout,

@@ -147,3 +147,25 @@ def test_host_buffer_entry_point_matches_oracle(kind):
                       s.ws, s.compute)
         s.compute.synchronize()
         check_tolerance(_bits(yh), y_ref, what="host entry point")
+
+
+@pytest.mark.parametrize("rank,r_max", [(16, 16), (8, 16)])
+def test_packed_adapter_lands_in_the_slot_layout(rank, r_max):
+    """One pinned buffer per adapter (LORA_PACKED): the slot holds the same bytes as after a
+    matrix-by-matrix load, padding rows are zero, and the forward matches the oracle."""
+    from paper_2602_24044_b200 import binding as lb
+    from paper_2602_24044_b200.harness import Session
+    wl = W.make_custom(96, 256, 512, 4, rank, r_max=r_max, scale=0.7, index="uniform", seed=21)
+    wl.targets = wl.targets + [(512, 128)]
+    y_ref, _ = oracle_full(wl)
+    with Session(wl, slots=[]) as s:
+        for slot in range(4):
+            s.load_slot(slot, a_layout=lb.PACKED)
+        lb.pool_acquire(s.pool, list(range(4)), s.compute)
+        for slot in range(4):
+            for t in range(2):
+                A, B = s.read_slot(slot, t)
+                a, b = wl.adapter_weights(slot, t)
+                assert np.array_equal(A[:rank], a.T) and np.array_equal(B[:rank], b)
+                assert not A[rank:].any() and not B[rank:].any()
+        check_tolerance(_bits(s.apply()), y_ref, what="packed load")
