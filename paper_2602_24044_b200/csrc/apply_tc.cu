@@ -309,12 +309,16 @@ tc_shrink_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_x,
 // ---------------------------------------------------------------------------------------------
 template <int RP>
 struct ExpandCfg {
+#ifdef LORA_TC_EXPAND_STAGES
+    static constexpr int STAGES = LORA_TC_EXPAND_STAGES;
+#else
     static constexpr int STAGES = RP == 64 ? 4 : 6;
+#endif
     static constexpr int BT_BYTES = RP * 128;                       // RP rank rows x 64 columns
     static constexpr int STAGE = XT_BYTES + ((BT_BYTES + 1023) & ~1023);   // y_base/out tile + B tile
     static constexpr int V_BYTES = TC_ROWS * RP * 2;                // one bf16 copy of v
     static constexpr int SMEM = 2 * V_BYTES + STAGES * STAGE + 256 + 1024;
-    static constexpr uint32_t TMEM_COLS = STAGES == 4 ? 256 : 512;  // ring of 64-column accumulators
+    static constexpr uint32_t TMEM_COLS = STAGES <= 2 ? 128 : STAGES <= 4 ? 256 : 512;  // ring of 64-column accumulators
 };
 
 template <int RP>

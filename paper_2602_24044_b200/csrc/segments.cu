@@ -214,10 +214,246 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
     }
 }
 
+// The same table for long batches (prefill): the token list is cut into chunks and the position
+// of every token inside its slot's run comes from per-chunk, per-slot counts, so the work per block
+// is O(T) instead of O(T) per occupied slot.  Every block builds the small tables in shared memory
+// (counts, prefix sums, first and last token of every tile); the writes to global memory are
+// divided: a block writes the perm entries of its own chunks and the records of its own slots.
+// Tokens without an occupied slot are counted in an extra column and land behind the active ones.
+__global__ void __launch_bounds__(SEG_THREADS)
+build_segments_chunked_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int32_t T,
+                              int32_t tile_m, int32_t long_min, int32_t *meta, int32_t CH, int32_t C) {
+    extern __shared__ int32_t sm[];
+    const int32_t N = pool.num_slots, N1 = N + 1;
+    const MetaLayout L = meta_layout(T, N, tile_m);
+    int32_t *cnt = sm;             // [N] tokens per slot
+    int32_t *start = cnt + N;      // [N] first position in perm
+    int32_t *segid = start + N;    // [N] segment number
+    int32_t *tile0 = segid + N;    // [N] first tile number
+    int32_t *occ = tile0 + N;      // [N] slot occupied
+    int32_t *piece0 = occ + N;     // [N] first unit number
+    int32_t *tok = piece0 + N;     // [T] the token list
+    int32_t *cnt2 = tok + T;       // [C][N + 1] per chunk and slot: count, then running position
+    int32_t *tfirst = cnt2 + (int64_t)C * N1;   // [cap_tile] first token id of a tile
+    int32_t *tlast = tfirst + L.cap_tile;       // [cap_tile] last token id of a tile
+    __shared__ int32_t warp_tot[4][SEG_WARPS];
+    __shared__ int32_t totals[4];
+    __shared__ int32_t n_invalid_s;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    for (int32_t s = tid; s < N; s += SEG_THREADS) {
+        cnt[s] = 0;
+        occ[s] = pool.table[s].loaded;
+    }
+    for (int32_t i = tid; i < C * N1; i += SEG_THREADS) cnt2[i] = 0;
+    for (int32_t t = tid; t < T; t += SEG_THREADS) tok[t] = slot_idx_g[t];
+    if (tid == 0) n_invalid_s = 0;
+    __syncthreads();
+
+    // column of a token: its slot when that is occupied, else the extra column N
+    auto classify = [&](int32_t t, int32_t t1, int32_t &s, bool &valid, bool &act) {
+        valid = t < t1;
+        s = valid ? tok[t] : -1;
+        act = valid && s >= 0 && s < N && occ[s];
+        return valid ? (act ? s : N) : -1 - lane;   // distinct keys for lanes past the end
+    };
+
+    // ---- 1. counts per chunk and column --------------------------------------------------------
+    for (int32_t c = warp; c < C; c += SEG_WARPS) {
+        const int32_t t0 = c * CH, t1 = min(T, t0 + CH);
+        for (int32_t base = t0; base < t1; base += 32) {
+            int32_t s; bool valid, act;
+            const int32_t col = classify(base + lane, t1, s, valid, act);
+            const uint32_t peers = __match_any_sync(0xffffffffu, col);
+            if (valid && lane == __ffs(peers) - 1) cnt2[c * N1 + col] += __popc(peers);
+            const uint32_t bad = __ballot_sync(0xffffffffu, valid && !act && s != -1);
+            if (lane == 0 && bad) atomicAdd(&n_invalid_s, __popc(bad));
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+    // ---- 2. per column: exclusive prefix over the chunks; per slot: totals and prefix sums -------
+    for (int32_t col = tid; col < N1; col += SEG_THREADS) {
+        int32_t run = 0;
+        for (int32_t c = 0; c < C; ++c) {
+            const int32_t v = cnt2[c * N1 + col];
+            cnt2[c * N1 + col] = run;
+            run += v;
+        }
+        if (col < N) cnt[col] = run;
+    }
+    __syncthreads();
+    const int32_t per = (N + SEG_THREADS - 1) / SEG_THREADS;
+    const int32_t lo = min(tid * per, N), hi = min(lo + per, N);
+    const int32_t ppt = (tile_m + 15) / 16;
+    auto pieces_of = [&](int32_t n) { return (n / tile_m) * ppt + ((n % tile_m) + 15) / 16; };
+    int32_t c_ = 0, z = 0, tl = 0, pc = 0;
+    for (int32_t s = lo; s < hi; ++s) {
+        c_ += cnt[s];
+        z += cnt[s] > 0;
+        tl += (cnt[s] + tile_m - 1) / tile_m;
+        pc += pieces_of(cnt[s]);
+    }
+    int32_t ic = c_, iz = z, it = tl, ip = pc;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int32_t a = __shfl_up_sync(0xffffffffu, ic, o);
+        const int32_t b = __shfl_up_sync(0xffffffffu, iz, o);
+        const int32_t d = __shfl_up_sync(0xffffffffu, it, o);
+        const int32_t e = __shfl_up_sync(0xffffffffu, ip, o);
+        if (lane >= o) { ic += a; iz += b; it += d; ip += e; }
+    }
+    if (lane == 31) {
+        warp_tot[0][warp] = ic; warp_tot[1][warp] = iz; warp_tot[2][warp] = it; warp_tot[3][warp] = ip;
+    }
+    __syncthreads();
+    int32_t bc = 0, bz = 0, bt = 0, bp = 0;
+    for (int w = 0; w < warp; ++w) {
+        bc += warp_tot[0][w]; bz += warp_tot[1][w]; bt += warp_tot[2][w]; bp += warp_tot[3][w];
+    }
+    int32_t rc = bc + ic - c_, rz = bz + iz - z, rt = bt + it - tl, rp = bp + ip - pc;
+    for (int32_t s = lo; s < hi; ++s) {
+        start[s] = rc;
+        segid[s] = rz;
+        tile0[s] = rt;
+        piece0[s] = rp;
+        rc += cnt[s];
+        rz += cnt[s] > 0;
+        rt += (cnt[s] + tile_m - 1) / tile_m;
+        rp += pieces_of(cnt[s]);
+    }
+    if (tid == SEG_THREADS - 1) { totals[0] = rc; totals[1] = rz; totals[2] = rt; totals[3] = rp; }
+    __syncthreads();
+    const int32_t n_active = totals[0], n_seg = totals[1], n_tile = totals[2], n_piece = totals[3];
+
+    // ---- 3. position of every token; first and last token of every tile --------------------------
+    int32_t *perm = meta + L.perm;
+    for (int32_t c = warp; c < C; c += SEG_WARPS) {
+        const int32_t t0 = c * CH, t1 = min(T, t0 + CH);
+        const bool mine = (c % (int32_t)gridDim.x) == (int32_t)blockIdx.x;
+        for (int32_t base = t0; base < t1; base += 32) {
+            const int32_t t = base + lane;
+            int32_t s; bool valid, act;
+            const int32_t col = classify(t, t1, s, valid, act);
+            const uint32_t peers = __match_any_sync(0xffffffffu, col);
+            int32_t j = 0;
+            if (valid) j = cnt2[c * N1 + col] + __popc(peers & ((1u << lane) - 1u));
+            __syncwarp();
+            if (valid && lane == __ffs(peers) - 1) cnt2[c * N1 + col] += __popc(peers);
+            __syncwarp();
+            if (act) {
+                const int32_t k = j / tile_m, jj = j - k * tile_m, idx = tile0[s] + k;
+                if (jj == 0) tfirst[idx] = t;
+                if (jj == tile_m - 1 || j == cnt[s] - 1) tlast[idx] = t;
+                if (mine) {
+                    perm[start[s] + j] = t;
+                    meta[L.unit_perm + 16 * (int64_t)(piece0[s] + k * ppt + (jj >> 4)) + (jj & 15)] = t;
+                }
+            } else if (valid && mine) {
+                perm[n_active + j] = t;
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- 4. segment, tile and unit records of this block's slots ---------------------------------
+    for (int32_t s = blockIdx.x * SEG_WARPS + warp; s < N; s += gridDim.x * SEG_WARPS) {
+        const int32_t n = cnt[s];
+        if (n == 0) continue;
+        const int32_t p0 = start[s], seg = segid[s];
+        const int32_t nt = (n + tile_m - 1) / tile_m;
+        const SlotEntry e = pool.table[s];
+        if (lane == 0) {
+            const int32_t first = tfirst[tile0[s]], last = tlast[tile0[s] + nt - 1];
+            meta[L.seg_slot + seg] = s;
+            meta[L.seg_start + seg] = p0;
+            meta[L.seg_rank + seg] = e.rank;
+            meta[L.seg_flags + seg] = (last - first + 1 == n ? 1 : 0) | (n >= long_min ? 2 : 0);
+        }
+        for (int32_t k = lane; k < nt; k += 32) {
+            const int32_t r0 = p0 + k * tile_m;
+            const int32_t rows = min(tile_m, p0 + n - r0);
+            const int32_t idx = tile0[s] + k;
+            meta[L.tile_seg + idx] = seg;
+            meta[L.tile_row0 + idx] = r0;
+            meta[L.tile_rows + idx] = rows;
+            const int32_t contiguous = (tlast[idx] - tfirst[idx] + 1 == rows) ? 1 : 0;
+            meta[L.tile_flags + idx] = contiguous;
+            *reinterpret_cast<int4 *>(meta + L.tile_desc + 4 * (int64_t)idx) =
+                make_int4(s, r0, rows | (contiguous << 15) | (e.rank << 16), __float_as_int(e.scale));
+            for (int32_t i = 0; i < (rows + 15) / 16; ++i)
+                *reinterpret_cast<int4 *>(meta + L.unit_desc + 4 * (int64_t)(piece0[s] + k * ppt + i)) =
+                    make_int4(s, r0 + 16 * i,
+                              min(16, rows - 16 * i) | (rows << 8) | (contiguous << 16) | (e.rank << 17),
+                              __float_as_int(e.scale));
+        }
+    }
+
+    // ---- 5. last block: header, -1 in unused entries ---------------------------------------------
+    if (blockIdx.x != gridDim.x - 1) return;
+    if (tid == 0) {
+        const int32_t n_invalid = n_invalid_s;
+        meta[H_T] = T;
+        meta[H_NACTIVE] = n_active;
+        meta[H_NINVALID] = n_invalid;
+        meta[H_NSEG] = n_seg;
+        meta[H_NTILE] = n_tile;
+        meta[H_TILE_M] = tile_m;
+        meta[H_LONG_MIN] = long_min;
+        meta[H_NSLOTS] = N;
+        meta[H_CAP_SEG] = L.cap_seg;
+        meta[H_CAP_TILE] = L.cap_tile;
+        meta[H_NPIECE] = n_piece;
+        for (int i = H_NPIECE + 1; i < META_HEADER_WORDS; ++i) meta[i] = 0;
+        meta[L.seg_start + n_seg] = n_active;
+        if (n_invalid) atomicAdd(&pool.status[STATUS_INVALID_TOKENS], n_invalid);
+    }
+    for (int32_t i = n_seg + tid; i < L.cap_seg; i += SEG_THREADS) {
+        meta[L.seg_slot + i] = -1;
+        meta[L.seg_rank + i] = -1;
+        meta[L.seg_flags + i] = -1;
+    }
+    for (int32_t i = n_seg + 1 + tid; i <= L.cap_seg; i += SEG_THREADS) meta[L.seg_start + i] = -1;
+    for (int32_t i = n_tile + tid; i < L.cap_tile; i += SEG_THREADS) {
+        meta[L.tile_seg + i] = -1;
+        meta[L.tile_row0 + i] = -1;
+        meta[L.tile_rows + i] = -1;
+        meta[L.tile_flags + i] = -1;
+        *reinterpret_cast<int4 *>(meta + L.tile_desc + 4 * (int64_t)i) = make_int4(-1, 0, 0, 0);
+    }
+}
+
 lora_status_t launch_build_segments(lora_pool_t *pool, const int32_t *slot_idx_dev, int32_t T,
                                     int32_t tile_m, int32_t long_min, void *meta_dev,
                                     cudaStream_t stream) {
     const int32_t N = pool->num_slots;
+    // long batches: the chunked kernel, when its tables fit in shared memory
+    if (T >= 1024 && pool->tuning[7] != 1) {
+        int32_t CH = ((T + 63) / 64 + 31) & ~31;   // about 64 chunks, multiples of 32 tokens
+        if (CH < 128) CH = 128;
+        const int32_t C = (T + CH - 1) / CH;
+        const MetaLayout L = meta_layout(T, N, tile_m);
+        const size_t words = 6 * (size_t)N + (size_t)T + (size_t)C * (N + 1) + 2 * (size_t)L.cap_tile;
+        if (words * sizeof(int32_t) <= 200 * 1024) {
+            const size_t smem = words * sizeof(int32_t);
+            static size_t attr_chunked = 48 * 1024;
+            if (smem > attr_chunked) {
+                cudaError_t e = cudaFuncSetAttribute(build_segments_chunked_kernel,
+                                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                if (e != cudaSuccess) return cuda_fail(e);
+                attr_chunked = smem;
+            }
+            int grid = (N + SEG_WARPS - 1) / SEG_WARPS;
+            if (grid < (C + SEG_WARPS - 1) / SEG_WARPS) grid = (C + SEG_WARPS - 1) / SEG_WARPS;
+            if (grid > pool->sm_count) grid = pool->sm_count;
+            build_segments_chunked_kernel<<<grid, SEG_THREADS, smem, stream>>>(
+                pool->view(), slot_idx_dev, T, tile_m, long_min, (int32_t *)meta_dev, CH, C);
+            return count_launch();
+        }
+    }
     int grid = (N + SEG_WARPS - 1) / SEG_WARPS;
     if (grid > 2 * pool->sm_count) grid = 2 * pool->sm_count;
     if (grid < 1) grid = 1;

@@ -59,6 +59,31 @@ def test_segments_bit_exact(case, tile_m):
         assert s.status()[0] == ref["header"][2]
 
 
+@pytest.mark.parametrize("tile_m", [1, 16, 100, 128])
+@pytest.mark.parametrize("case", ["uniform", "sorted", "zipf", "invalid", "same", "none"])
+def test_segments_bit_exact_long_batches(case, tile_m):
+    """Batches of 1024 tokens and more take the chunk-parallel builder: same table, bit for bit."""
+    kw = dict(T=4999, d_in=64, d_out=64, num_slots=53, ranks=[8, 16, 4, 32], unloaded=(5, 17))
+    if case == "uniform":
+        kw.update(index="uniform", frac_none=0.05, T=1024)
+    elif case == "sorted":
+        kw.update(index="sorted")
+    elif case == "zipf":
+        kw.update(index="zipf", T=7777)
+    elif case == "invalid":
+        kw.update(frac_invalid=0.2, frac_none=0.2, T=3001)
+    elif case == "same":
+        kw.update(index="same", T=2048)
+    elif case == "none":
+        kw.update(frac_none=1.0, T=1500)
+    wl = W.make_custom(**kw)
+    with _session(wl) as s:
+        s.build_segments(tile_m=tile_m, long_min=64)
+        got = s.segments_host()
+        ref = check_segments(got, wl, tile_m, 64)
+        assert s.status()[0] == ref["header"][2]
+
+
 @pytest.mark.parametrize("cfg", [0, 1, 2, 3])
 def test_segments_on_configs(cfg):
     wl = W.make_config(cfg)
