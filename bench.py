@@ -31,6 +31,10 @@ ROTATION = 16          # independent input / weight sets cycled through so every
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (None: no capture of the current kernel on that workload)
+NCU_TRAFFIC = {1: 22.9e6}
+
 PAPER_CONTEXT = {
     "note": "system-level results of the paper, other hardware, context only",
     "dt_throughput_smape": "2.25-5.08 % (Digital Twin on 1 CPU core vs vLLM v0.8.5 on 1x H100 64 GB)",
@@ -471,7 +475,7 @@ def main():
             "kernel": ("fused_kernel (one launch per apply and rank bucket)" if fused
                        else "shrink_kernel + expand_kernel (two launches per apply)"),
             "algorithmic_bytes_per_launch": alg / calls_per_step,
-            "us_per_launch": apply_ms * 1e3, "traffic": None,
+            "us_per_launch": apply_ms * 1e3, "traffic": NCU_TRAFFIC.get(cfg) if fused else None,
             "averaged_over": "%d applies per step" % calls_per_step,
         },
         "step_GBps": alg / (ms / K * 1e-3) / 1e9,

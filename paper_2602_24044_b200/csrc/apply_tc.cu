@@ -569,6 +569,11 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
                                    size_t workspace_bytes, cudaStream_t stream, bool *handled) {
     *handled = false;
     if (!AP.meta || AP.tile_m != TC_ROWS || AP.T < TC_ROWS) return LORA_OK;
+    // Fewer than ~32 full tiles cannot fill the GPU with 128-row blocks (the grids below are sized
+    // by a bound on the tile count, not the count itself); the fused kernel alone was measured
+    // faster there (mixed chunked-prefill batch: 108 us against 166 us).  Tuning key 4 = 2 forces
+    // this path whenever it applies.
+    if (AP.T / TC_ROWS < 32 && pool->tuning[4] != 2) return LORA_OK;
     if (!encode_fn()) return LORA_OK;
     // TMA wants 16-byte aligned bases and row pitches
     if ((((uintptr_t)AP.x | (uintptr_t)AP.yb | (uintptr_t)AP.y) & 15) || (AP.ldx % 8) || (AP.ldyb % 8) ||

@@ -17,6 +17,8 @@ def _gpu():
 def _run(wl, tuning=None, **kw):
     from paper_2602_24044_b200 import binding as lb
     from paper_2602_24044_b200.harness import Session, bf16_bits
+    if tuning is None:
+        tuning = {4: 2}   # these batches are short: force the tensor-core kernels wherever they apply
     with Session(wl, tuning=tuning) as s:
         before = lb.launch_count()
         y = bf16_bits(s.apply(**kw))
