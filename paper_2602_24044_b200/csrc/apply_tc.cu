@@ -59,6 +59,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1,
                                             uint64_t *bar) {
     asm volatile(
@@ -154,6 +157,7 @@ __host__ __device__ constexpr uint32_t instr_desc(uint32_t M, uint32_t N, uint32
 }  // namespace tc
 
 constexpr int TC_THREADS = 128;
+constexpr int TCX_THREADS = 160;   // expand: four epilogue warps and one warp that issues copies and MMAs
 constexpr int TC_ROWS = 128;       // rows of a long tile
 constexpr int SH_STAGES = 4;       // shrink: ring of (x tile, A tile) stages
 constexpr int XT_BYTES = TC_ROWS * 128;   // 128 rows x 64 bf16
@@ -322,7 +326,7 @@ struct ExpandCfg {
 };
 
 template <int RP>
-__global__ void __launch_bounds__(TC_THREADS)
+__global__ void __launch_bounds__(TCX_THREADS)
 tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
                  const __grid_constant__ CUtensorMap map_yb, const __grid_constant__ CUtensorMap map_y) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -336,7 +340,9 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
     unsigned char *Vl = Vh + C::V_BYTES;
     uint64_t *full = reinterpret_cast<uint64_t *>(Vl + C::V_BYTES);
     uint64_t *mma_done = full + S;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(mma_done + S);
+    uint64_t *freed = mma_done + S;     // the epilogue is done with a stage and its store has read it
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(freed + S);
+    volatile int32_t *failed = reinterpret_cast<volatile int32_t *>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const LongTile lt = long_tile(P, blockIdx.x);
@@ -349,17 +355,22 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
     if (nblk <= 0) return;
 
     if (tid == 0) {
-        for (int s = 0; s < S; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&mma_done[s], 1); }
+        for (int s = 0; s < S; ++s) {
+            tc::mbar_init(&full[s], 1);
+            tc::mbar_init(&mma_done[s], 1);
+            tc::mbar_init(&freed[s], 1);
+        }
+        *failed = 0;
         tc::fence_mbar_init();
     }
-    if (warp == 0) {
+    if (warp == 4) {
         tc::tmem_alloc(tmem_slot, C::TMEM_COLS);
         tc::tmem_relinquish();
     }
     // v = sum of the K-slice partials (in order); thread = row.  Stored as bf16 high and low parts
     // in the no-swizzle K-major layout: 8 x 8 core matrices of 128 bytes, the core matrix of row
     // group mg and rank group kg at (kg * 16 + mg) * 128 bytes.
-    {
+    if (tid < TC_ROWS) {
         const int32_t m = tid;
         const float *src = P.ws + ((int64_t)lt.row0 + m) * P.RS;
         const int64_t ks_stride = (int64_t)P.T * P.RS;
@@ -421,68 +432,91 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
         return true;
     };
 
-    if (tid == 0) {
-        for (int32_t j = 0; j < nblk && j < S - 1; ++j) issue_load(j);
-        ok = issue_mma(0);
-    }
-    for (int32_t j = 0; j < nblk; ++j) {
-        const int s = j % S;
-        if (tid == 0 && ok && j + 1 < nblk) ok = issue_mma(j + 1);   // next block's MMAs run under this epilogue
-        ok = __syncthreads_and(ok ? 1 : 0) != 0;
-        if (!ok) break;
-        if (!tc::mbar_wait(&mma_done[s], (uint32_t)(j / S) & 1u)) ok = false;
-        tc::tc_fence_after();
-        // epilogue: thread = row; the y_base tile (128-byte swizzle) is updated in place
-        unsigned char *tile = stages + s * C::STAGE;
+    if (warp == 4) {
+        // ---- producer: one thread requests tiles S - 2 blocks ahead and issues each block's MMAs
+        // as soon as its tiles have landed; it never waits for an epilogue that is under way ------
+        if (lane == 0) {
+            for (int32_t j = 0; j < nblk && j < S - 2; ++j) issue_load(j);
+            for (int32_t j = 0; j < nblk && ok; ++j) {
+                if (*failed) break;
+                ok = issue_mma(j);
+                const int32_t n = j + S - 2;          // next block to request
+                if (ok && n < nblk) {
+                    if (n >= S) ok = tc::mbar_wait(&freed[n % S], (uint32_t)(n / S - 1) & 1u);
+                    if (ok) issue_load(n);
+                }
+            }
+            if (!ok) *failed = 1;
+        }
+        __syncwarp();
+    } else {
+        // ---- epilogue warps: thread = row; the y_base tile (128-byte swizzle) is updated in place
         const int m = warp * 32 + lane;
+        for (int32_t j = 0; j < nblk; ++j) {
+            const int s = j % S;
+            // all four warps take the same decision (a thread that left alone would strand the
+            // others at the named barrier below)
+            const uint32_t bad = (*failed != 0 || !tc::mbar_wait(&mma_done[s], (uint32_t)(j / S) & 1u)) ? 1u : 0u;
+            uint32_t any_bad;
+            asm volatile(
+                "{\n\t.reg .pred p, q;\n\t"
+                "setp.ne.u32 p, %1, 0;\n\t"
+                "bar.red.or.pred q, 1, 128, p;\n\t"
+                "selp.u32 %0, 1, 0, q;\n\t}"
+                : "=r"(any_bad)
+                : "r"(bad)
+                : "memory");
+            if (any_bad) { ok = false; *failed = 1; break; }
+            tc::tc_fence_after();
+            unsigned char *tile = stages + s * C::STAGE;
 #pragma unroll
-        for (int c = 0; c < 64; c += 16) {
-            uint32_t r[16];
-            tc::tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + s * 64 + c, r);
-            tc::tmem_ld_wait();
+            for (int c = 0; c < 64; c += 16) {
+                uint32_t r[16];
+                tc::tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + s * 64 + c, r);
+                tc::tmem_ld_wait();
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int chunk = (c >> 3) + h;
-                uint4 *p = reinterpret_cast<uint4 *>(tile + m * 128 + ((chunk ^ (m & 7)) << 4));
-                float acc[8];
+                for (int h = 0; h < 2; ++h) {
+                    const int chunk = (c >> 3) + h;
+                    uint4 *p = reinterpret_cast<uint4 *>(tile + m * 128 + ((chunk ^ (m & 7)) << 4));
+                    float acc[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[e] = __uint_as_float(r[h * 8 + e]);
-                *p = finish8(acc, *p, lt.scale);
+                    for (int e = 0; e < 8; ++e) acc[e] = __uint_as_float(r[h * 8 + e]);
+                    *p = finish8(acc, *p, lt.scale);
+                }
+            }
+            tc::tc_fence_before();
+            if (lt.rows < TC_ROWS) {
+                // short tile: the rows after it belong to other tokens, so each thread stores its own row
+                const int32_t colb = (b0 + j) * 64;
+                if (m < lt.rows) {
+                    __nv_bfloat16 *yrow = P.y + (int64_t)(lt.t0 + m) * P.ldy + colb;
+#pragma unroll
+                    for (int chunk = 0; chunk < 8; ++chunk)
+                        if (colb + chunk * 8 < P.tv.d_out)
+                            *reinterpret_cast<uint4 *>(yrow + chunk * 8) =
+                                *reinterpret_cast<const uint4 *>(tile + m * 128 + ((chunk ^ (m & 7)) << 4));
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");   // every row has left the stage
+                if (tid == 0) tc::mbar_arrive(&freed[s]);
+            } else {
+                tc::fence_proxy_async();    // the tile is read by the TMA store
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (tid == 0) {
+                    tc::tma_store_2d(&map_y, (b0 + j) * 64, lt.t0, tile);
+                    tc::bulk_commit();
+                    if (j > 0) {
+                        tc::bulk_wait_read<1>();      // the store before this one has read its stage
+                        tc::mbar_arrive(&freed[(j - 1) % S]);
+                    }
+                }
             }
         }
-        tc::fence_proxy_async();    // the tile is read by the TMA store
-        tc::tc_fence_before();
-        ok = __syncthreads_and(ok ? 1 : 0) != 0;
-        if (!ok) break;
-        if (lt.rows < TC_ROWS) {
-            // short tile: the rows after it belong to other tokens, so each thread stores its own row
-            const int32_t colb = (b0 + j) * 64;
-            if (m < lt.rows) {
-                __nv_bfloat16 *yrow = P.y + (int64_t)(lt.t0 + m) * P.ldy + colb;
-#pragma unroll
-                for (int chunk = 0; chunk < 8; ++chunk)
-                    if (colb + chunk * 8 < P.tv.d_out)
-                        *reinterpret_cast<uint4 *>(yrow + chunk * 8) =
-                            *reinterpret_cast<const uint4 *>(tile + m * 128 + ((chunk ^ (m & 7)) << 4));
-            }
-        }
-        if (tid == 0) {
-            if (lt.rows == TC_ROWS) tc::tma_store_2d(&map_y, (b0 + j) * 64, lt.t0, tile);
-            tc::bulk_commit();
-            const int32_t n = j + S - 1;          // next block to request: into the stage used by block j - 1
-            if (n < nblk) {
-                tc::bulk_wait_read<1>();          // that stage's store has finished reading shared memory
-                issue_load(n);
-            }
-        }
+        if (tid == 0) tc::bulk_wait_read<0>();
     }
-    if (tid == 0) {
-        tc::bulk_wait_read<0>();
-        if (!ok) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
-    }
+    if (tid == 0 && *failed) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
     tc::tc_fence_before();
     __syncthreads();
-    if (warp == 0) tc::tmem_dealloc(tmem, C::TMEM_COLS);
+    if (warp == 4) tc::tmem_dealloc(tmem, C::TMEM_COLS);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -558,7 +592,7 @@ static lora_status_t launch_tc_bucket(lora_pool_t *pool, const TcParams &P, cons
     tc_shrink_kernel<RP><<<dim3(units, P.KS), TC_THREADS, SH_SMEM, stream>>>(P, mx, ma);
     lora_status_t s = count_launch();
     if (s != LORA_OK) return s;
-    tc_expand_kernel<RP><<<dim3(units, P.NS), TC_THREADS, ExpandCfg<RP>::SMEM, stream>>>(P, mb, myb, my);
+    tc_expand_kernel<RP><<<dim3(units, P.NS), TCX_THREADS, ExpandCfg<RP>::SMEM, stream>>>(P, mb, myb, my);
     return count_launch();
 }
 
