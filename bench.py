@@ -472,8 +472,9 @@ def main():
             "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
             "frac": achieved / peak, "peak_source": "%s copy bandwidth" % peak_kind,
             "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-            "kernel": ("fused_kernel (one launch per apply and rank bucket)" if fused
-                       else "shrink_kernel + expand_kernel (two launches per apply)"),
+            "kernel": ("shrink_kernel + expand_kernel (two launches per apply)" if not fused
+                       else "tc_shrink_kernel + tc_expand_kernel + fused_kernel (one apply; tc_expand dominates)"
+                       if cfg == 2 else "fused_kernel (one launch per apply, every rank)"),
             "algorithmic_bytes_per_launch": alg / calls_per_step,
             "us_per_launch": apply_ms * 1e3, "traffic": NCU_TRAFFIC.get(cfg) if fused else None,
             "averaged_over": "%d applies per step" % calls_per_step,

@@ -316,7 +316,7 @@ struct ExpandCfg {
 #ifdef LORA_TC_EXPAND_STAGES
     static constexpr int STAGES = LORA_TC_EXPAND_STAGES;
 #else
-    static constexpr int STAGES = RP == 64 ? 4 : 6;
+    static constexpr int STAGES = 4;   // 2 blocks per SM up to rank 32; deeper rings measured slower
 #endif
     static constexpr int BT_BYTES = RP * 128;                       // RP rank rows x 64 columns
     static constexpr int STAGE = XT_BYTES + ((BT_BYTES + 1023) & ~1023);   // y_base/out tile + B tile
