@@ -532,7 +532,13 @@ fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
     // stream is still running.  Activations are only touched after griddep_wait().  The unit
     // records and the pool were complete before that kernel started when P.early is set (the host
     // sets it only then), so they are read, and the first weight tiles requested, ahead of the wait.
-    if (!P.early) griddep_wait();
+    if (!P.early) {
+        // nothing may be read yet: use the time for the zeros in every stage (rows above a unit's
+        // rank are never copied, and what they hold is multiplied by zeros of v, so it has to be finite)
+        for (int i = tid; i < P.n_stages * P.stage_bytes / 16; i += FT)
+            reinterpret_cast<uint4 *>(smem + P.off_stage)[i] = make_uint4(0, 0, 0, 0);
+        griddep_wait();
+    }
     {
         // the number of units and the records of this cluster's first two units, side by side
         UnitRegs m0, m1;
@@ -541,10 +547,10 @@ fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
             m1 = fetch_unit(P, cx.cid + cx.G, P.units, lane);
         }
         cx.n_units = P.meta ? ldg_int(P.meta + H_NPIECE) : P.T;
-        // meanwhile: zeros in every stage (rows above a unit's rank are never copied, and what
-        // they hold is multiplied by zeros of v, so it has to be finite)
-        for (int i = tid; i < P.n_stages * P.stage_bytes / 16; i += FT)
-            reinterpret_cast<uint4 *>(smem + P.off_stage)[i] = make_uint4(0, 0, 0, 0);
+        // meanwhile (early mode): the zeros in every stage
+        if (P.early)
+            for (int i = tid; i < P.n_stages * P.stage_bytes / 16; i += FT)
+                reinterpret_cast<uint4 *>(smem + P.off_stage)[i] = make_uint4(0, 0, 0, 0);
         fence_proxy_async();   // the stages are written by bulk copies from here on
         if (cx.n_units > P.units) cx.n_units = P.units;
         if (warp == 3) {
@@ -724,7 +730,9 @@ static lora_status_t launch_h(lora_pool_t *pool, ApplyParams P, int32_t C, const
     // ordered behind the build, so the table is complete before this kernel can start.
     const bool fresh = P.meta ? pool->take_fresh(P.meta) : true;
     P.early = (P.meta && !fresh && pool->tuning[2] != 2) ? 1 : 0;
-    const unsigned n_attrs = P.early ? 2 : 1;
+    // Without `early` the attribute still lets the blocks become resident and set up their shared
+    // memory while the kernel before them drains; they read nothing until it has completed.
+    const unsigned n_attrs = pool->tuning[2] != 2 ? 2 : 1;
 
     // Grid: no more clusters than can be resident at once (each loops over its units), so no
     // cluster of an over-sized grid waits for a slot only to find that its unit does not exist.

@@ -265,3 +265,33 @@ def test_layer_step_config_all_projections():
             y_ref, _ = oracle_full(wl, call)
             y = s.apply(call, rebuild=(call == 0))
             check_tolerance(_bits(y), y_ref, what="config 4 projection %d" % call)
+
+
+def test_back_to_back_applies_on_one_table():
+    """Several applies queued behind one metadata build, without a host synchronisation between
+    them: from the second on, the kernels may read the table and the pool before their predecessor
+    has finished (programmatic dependent launch).  Every result must still match the oracle."""
+    from paper_2602_24044_b200 import binding as lb
+    from paper_2602_24044_b200.harness import bf16_tensor
+    import torch
+    wl = W.make_custom(200, 1024, 768, 24, [8, 16, 16, 32], scale=0.7, index="zipf", tile_m=8,
+                       weight_mode="unitB", frac_none=0.05, seed=77)
+    wl.targets = wl.targets * 3
+    wl.calls = [0, 1, 2]
+    with _session(wl) as s:
+        s.build_segments()
+        outs = []
+        for c in range(3):
+            x_h, yb_h = wl.activations(c)
+            x, yb = bf16_tensor(x_h, s.device), bf16_tensor(yb_h, s.device)
+            y = torch.empty_like(yb)
+            outs.append((x, yb, y))
+        for rep in range(2):            # second round: every launch is of the early kind
+            for c, (x, yb, y) in enumerate(outs):
+                lb.bgmv_apply(s.pool, c, x, x.shape[1], yb, yb.shape[1], y, y.shape[1], s.slot_idx_dev,
+                              wl.T, s.meta, s.ws, stream=s.compute)
+        torch.cuda.synchronize()
+        for c, (x, yb, y) in enumerate(outs):
+            y_ref, _ = oracle_full(wl, call=c)
+            check_tolerance(_bits(y), y_ref, what="apply %d of 3 on one table" % c)
+        assert s.status()[1] == 0
