@@ -416,15 +416,28 @@ def main():
     ybh = [bf16_tensor(yb_h, pin=True) for _ in range(2)]
     yh = [torch.empty((T, d_out0), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
     sh = torch.from_numpy(wl.slot_idx.copy()).pin_memory()
-    sd = torch.empty(T, dtype=torch.int32, device=dev)
-    tp0, xd, ybd, yd = sets[0][0]
+    tp0, xd0, ybd0, yd0 = sets[0][0]
+    # two lanes (stream + device staging buffers each), used alternately: the host-to-device copy of
+    # one step overlaps the device-to-host copy of the step before it
+    lanes = []
+    for lane in range(2):
+        lanes.append({
+            "stream": s.compute if lane == 0 else torch.cuda.Stream(dev),
+            "x": xd0 if lane == 0 else torch.empty_like(xd0),
+            "yb": ybd0 if lane == 0 else torch.empty_like(ybd0),
+            "y": yd0 if lane == 0 else torch.empty_like(yd0),
+            "sidx": torch.empty(T, dtype=torch.int32, device=dev),
+            "meta": metas[0] if lane == 0 else torch.empty_like(metas[0]),
+            "ws": s.ws if lane == 0 else torch.empty_like(s.ws),
+        })
 
     def e2e_step(i):
         c = i % 2
+        L = lanes[c]
         lb.apply_host(s.pool, tp0, 1 if sgmv else 0, xh[c], ybh[c], yh[c], sh, T, wl.tile_m, wl.long_min,
-                      xd, ybd, yd, sd, metas[0], s.ws, s.compute)
+                      L["x"], L["yb"], L["y"], L["sidx"], L["meta"], L["ws"], L["stream"])
 
-    for i in range(3):
+    for i in range(4):
         e2e_step(i)
     torch.cuda.synchronize()
     if world > 1:
@@ -432,7 +445,8 @@ def main():
     t0 = time.perf_counter()
     for i in range(Ke):
         e2e_step(i)
-    s.compute.synchronize()
+    for L in lanes:
+        L["stream"].synchronize()
     e2e_s = time.perf_counter() - t0
     if world > 1:
         t = torch.tensor([e2e_s], device=dev)
@@ -481,7 +495,7 @@ def main():
         },
         "step_GBps": alg / (ms / K * 1e-3) / 1e9,
         "e2e": {"value": world * T * Ke / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "api": "lora_apply_host (first projection of the step)",
+                "d2h_bytes_per_step": d2h, "api": "lora_apply_host (first projection of the step), two streams used alternately",
                 "steps": Ke},
         "gpu_launches": int(launches),
         "clocks": clocks,

@@ -145,8 +145,15 @@ lora_status_t lora_pool_slot_info(const lora_pool_t *pool, int32_t slot, int32_t
 lora_status_t lora_pool_poll_status(lora_pool_t *pool, int32_t *host_out, void *stream);
 lora_status_t lora_pool_reset_status(lora_pool_t *pool, void *stream);
 
-/* Tuning knobs, for measurement.  key 0: apply algorithm (0 = default); see the library's
- * documentation for the values.  Unknown keys -> INVALID_ARG. */
+/* Tuning knobs, for measurement (0 = the default behaviour for every key):
+ *   key 0  apply path: 1 = two-phase CUDA-core kernels with the fp32 workspace
+ *   key 1  fused kernel: blocks per cluster (1, 2, 4, 8)
+ *   key 2  programmatic dependent launch of the fused kernel: 2 = never
+ *   key 3  fused kernel: upper bound on the clusters in the grid
+ *   key 4  tensor-core kernels of lora_sgmv_apply: 1 = never, 2 = whenever they apply
+ *   key 5  fused kernel: stages of the shared-memory ring (2 .. 4)
+ *   key 7  segment builder: 1 = one warp per slot also for long batches
+ * Keys outside 0 .. 7 -> INVALID_ARG. */
 lora_status_t lora_pool_set_tuning(lora_pool_t *pool, int32_t key, int32_t value);
 
 /* ----------------------------------------------------------------------------------------
@@ -184,8 +191,14 @@ lora_status_t lora_build_segments(lora_pool_t *pool, const int32_t *slot_idx_dev
  * not overlapping it.  Tokens without an active slot get y = y_base bit for bit.  Row t of y
  * depends only on row t of x and y_base, the token's slot and the pool.
  * workspace: dev scratch of >= lora_workspace_bytes(pool, T) bytes (fp32 partial products
- * v = x . A_i between the two phases), contents undefined afterwards; calls sharing a workspace
- * must be ordered on one stream.
+ * v = x . A_i between the two phases of the tensor-core and two-phase kernels; the fused kernel
+ * keeps v on chip), contents undefined afterwards; calls sharing a workspace must be ordered on
+ * one stream.
+ * Ordering: every apply is ordered behind the lora_build_segments call that wrote its table.
+ * Later applies on the same table may start reading the table and the pool (never x or y_base)
+ * while the kernel queued before them on the stream is still running, so nothing queued between
+ * two applies may write the table or the pool without an event or a rebuild in between (slot
+ * loads go through lora_pool_load_slot / lora_pool_acquire, which order themselves).
  * T == 0 returns LORA_OK without launching.
  * Errors: INVALID_ARG, SHAPE, SLOT_RANGE (target), BUFFER_TOO_SMALL, CUDA.
  * -------------------------------------------------------------------------------------- */
@@ -231,8 +244,9 @@ lora_status_t lora_bgmv_apply_static(lora_pool_t *pool, int32_t target,
                                      const void *meta_dev_or_null, void *stream);
 
 /* Prefill / chunked-prefill batches.  meta_dev: metadata built for this batch (any tile_m).
- * Full tiles of 128 consecutive tokens take the tensor-core path when the pool's tuning allows
- * it; all other tiles take the CUDA-core path. */
+ * With tile_m = 128 and a batch of at least 4096 tokens, tiles that are runs of 32 .. 128
+ * consecutive tokens take the tcgen05 kernels (split-K partials in `workspace`); every other tile,
+ * and every tile of a shorter batch, takes the fused kernel that also serves lora_bgmv_apply. */
 lora_status_t lora_sgmv_apply(lora_pool_t *pool, int32_t target,
                               const void *x, int64_t ldx,
                               const void *y_base, int64_t ldyb,

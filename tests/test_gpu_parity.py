@@ -295,3 +295,4 @@ def test_back_to_back_applies_on_one_table():
             y_ref, _ = oracle_full(wl, call=c)
             check_tolerance(_bits(y), y_ref, what="apply %d of 3 on one table" % c)
         assert s.status()[1] == 0
+
