@@ -62,6 +62,23 @@ def parse_args():
     return ap.parse_args()
 
 
+def max_over_ranks(value, device=None):
+    """The largest `value` of all ranks (every rank gets it); the identity without a process group."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world, tokens_per_step, steps, ms):
+    """Tokens per second of all replicas together: every rank ran `steps` steps of its own batch in
+    `ms` milliseconds (the slowest rank's time)."""
+    return world * tokens_per_step * steps / (ms * 1e-3)
+
+
 def measured_peak():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -364,11 +381,7 @@ def main():
     launches = (K // n_sets) * launches_per_rotation + (lb.launch_count() - l0)
     if world > 1:
         dist.barrier()
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(e0.elapsed_time(e1), dev)
 
     # the applies alone (dominant kernel), same rotation, for the roofline figure
     Kr = max(n_sets, min(K, 16000) // n_sets * n_sets)
@@ -447,11 +460,7 @@ def main():
         e2e_step(i)
     for L in lanes:
         L["stream"].synchronize()
-    e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = max_over_ranks(time.perf_counter() - t0, dev)
     h2d = 2 * T * (d_in0 + d_out0) + 4 * T
     d2h = 2 * T * d_out0
 
@@ -467,7 +476,7 @@ def main():
     achieved = alg / calls_per_step / (apply_ms * 1e-3) / 1e9
     fused = tuning.get(0) != 1
     line = {
-        "metric": METRIC, "value": world * T * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": whole_job_value(world, T, K, ms), "unit": UNIT, "n_gpus": world,
         "steps": K, "warmup": args.warmup, "ms_per_step": ms / K, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in/out, fp32 accumulate",
         "data": "synthetic",
@@ -494,7 +503,7 @@ def main():
             "averaged_over": "%d applies per step" % calls_per_step,
         },
         "step_GBps": alg / (ms / K * 1e-3) / 1e9,
-        "e2e": {"value": world * T * Ke / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": whole_job_value(world, T, Ke, e2e_s * 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "api": "lora_apply_host (first projection of the step), two streams used alternately",
                 "steps": Ke},
         "gpu_launches": int(launches),
