@@ -296,3 +296,53 @@ def test_back_to_back_applies_on_one_table():
             check_tolerance(_bits(y), y_ref, what="apply %d of 3 on one table" % c)
         assert s.status()[1] == 0
 
+
+def test_graph_replay_of_rotating_steps_matches_oracle():
+    """The launch configuration bench.py times: a CUDA graph of consecutive steps (metadata build +
+    grouped apply) over rotating copies of the config-1 projection, replayed several times.  Every
+    copy's result is compared with the oracle, and a replay must reproduce the first one bit for bit."""
+    import torch
+    from paper_2602_24044_b200 import binding as lb
+    from paper_2602_24044_b200.harness import bf16_tensor
+    wl = W.make_config(1)
+    R = 3
+    wl.targets = wl.targets * R
+    wl.calls = list(range(R))
+    with _session(wl, a_layout=lb.A_RANK_MAJOR) as s:
+        T = wl.T
+        nwords = lb.segments_bytes(T, wl.num_slots, wl.tile_m) // 4
+        sets, metas = [], []
+        for r in range(R):
+            x_h, yb_h = wl.activations(r)
+            x, yb = bf16_tensor(x_h, s.device), bf16_tensor(yb_h, s.device)
+            sets.append((x, yb, torch.empty_like(yb)))
+            metas.append(torch.empty(nwords, dtype=torch.int32, device=s.device))
+
+        def step(r):
+            x, yb, y = sets[r]
+            lb.build_segments(s.pool, s.slot_idx_dev, T, wl.tile_m, wl.long_min, metas[r], stream=s.compute)
+            lb.bgmv_apply(s.pool, r, x, x.shape[1], yb, yb.shape[1], y, y.shape[1], s.slot_idx_dev, T,
+                          metas[r], s.ws, stream=s.compute)
+
+        with torch.cuda.stream(s.compute):
+            for r in range(R):
+                step(r)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s.compute):
+            for r in range(R):
+                step(r)
+        with torch.cuda.stream(s.compute):
+            g.replay()
+        first = [_bits(sets[r][2]).copy() for r in range(R)]
+        for r in range(R):
+            sets[r][2].zero_()
+        with torch.cuda.stream(s.compute):
+            for _ in range(3):
+                g.replay()
+        for r in range(R):
+            y_ref, _ = oracle_full(wl, call=r)
+            got = _bits(sets[r][2])
+            check_tolerance(got, y_ref, what="graph replay, copy %d" % r)
+            assert np.array_equal(got, first[r])
+        assert s.status()[1] == 0
