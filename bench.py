@@ -161,7 +161,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def time_oracle(wl, budget_s=12.0, max_reps=2000, warm=1):
+def time_oracle(wl, budget_s=12.0, max_reps=20000, warm=1):
     """The CPU oracle as it stands on all host cores, on whole batches of the workload."""
     from oracle import lora_oracle as orc
     cores = orc.host_cores()
@@ -478,7 +478,7 @@ def main():
     line = {
         "metric": METRIC, "value": whole_job_value(world, T, K, ms), "unit": UNIT, "n_gpus": world,
         "steps": K, "warmup": args.warmup, "ms_per_step": ms / K, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in/out, fp32 accumulate",
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "accumulate": "fp32",
         "data": "synthetic",
         "config": {
             "workload": WORKLOAD_TEXT[cfg] + " (%d tokens, %d distinct adapters)" % (T, len(wl.distinct_slots())),
