@@ -346,3 +346,52 @@ def test_graph_replay_of_rotating_steps_matches_oracle():
             check_tolerance(got, y_ref, what="graph replay, copy %d" % r)
             assert np.array_equal(got, first[r])
         assert s.status()[1] == 0
+
+def test_two_layer_step_in_a_graph_with_swap_in_on_the_side_stream():
+    """Config 4 cut to two layers, run the way bench.py runs the 32-layer step: one metadata build
+    and 14 applies captured in a CUDA graph and replayed, while adapters that the step's tokens do
+    not use are swapped into their slots on the load stream.  All 14 outputs against the oracle."""
+    import torch
+    from paper_2602_24044_b200 import binding as lb
+    from paper_2602_24044_b200.harness import bf16_tensor
+    wl = W.make_config(4, layers=2)
+    n_calls = len(wl.calls)
+    with _session(wl, a_layout=lb.A_RANK_MAJOR) as s:
+        T = wl.T
+        meta = torch.empty(lb.segments_bytes(T, wl.num_slots, wl.tile_m) // 4, dtype=torch.int32,
+                           device=s.device)
+        bufs = []
+        for c in range(n_calls):
+            x_h, yb_h = wl.activations(c)
+            x, yb = bf16_tensor(x_h, s.device), bf16_tensor(yb_h, s.device)
+            bufs.append((x, yb, torch.empty_like(yb)))
+
+        def step():
+            lb.build_segments(s.pool, s.slot_idx_dev, T, wl.tile_m, wl.long_min, meta, stream=s.compute)
+            for c, (x, yb, y) in enumerate(bufs):
+                lb.bgmv_apply(s.pool, s.target_pos[wl.calls[c]], x, x.shape[1], yb, yb.shape[1], y,
+                              y.shape[1], s.slot_idx_dev, T, meta, s.ws, stream=s.compute)
+
+        with torch.cuda.stream(s.compute):
+            step()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s.compute):
+            step()
+        for _, _, y in bufs:
+            y.zero_()
+        victims = [int(v) for v in wl.swap_victims[:4]]
+        used = set(int(v) for v in wl.distinct_slots())
+        assert not used & set(victims)
+        blobs = [s.host_adapter_packed(v) for v in victims]
+        with torch.cuda.stream(s.compute):
+            g.replay()
+            for v, (A, B) in zip(victims, blobs):       # the same adapters again: contents unchanged
+                lb.pool_load_slot(s.pool, v, int(wl.ranks[v]), float(wl.scales[v]), A, B, lb.PACKED,
+                                  s.load, None, False)
+            g.replay()
+        torch.cuda.synchronize()
+        for c, (x, yb, y) in enumerate(bufs):
+            y_ref, _ = oracle_full(wl, c)
+            check_tolerance(_bits(y), y_ref, what="two-layer step, projection %d" % c)
+        assert s.status()[1] == 0
