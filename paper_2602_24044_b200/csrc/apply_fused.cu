@@ -708,10 +708,11 @@ static lora_status_t launch_h(lora_pool_t *pool, ApplyParams P, int32_t C, const
     P.n_stages = S;
     const int32_t smem = o;
 
-    static int32_t attr_smem = 0;
-    if (smem > attr_smem) {
+    const int dv = device_index(pool->device);
+    static int32_t attr_smem[DEVICE_TABLE] = {};
+    if (smem > attr_smem[dv]) {
         LORA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attr_smem = smem;
+        attr_smem[dv] = smem;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(FT, 1, 1);
@@ -736,7 +737,8 @@ static lora_status_t launch_h(lora_pool_t *pool, ApplyParams P, int32_t C, const
 
     // Grid: no more clusters than can be resident at once (each loops over its units), so no
     // cluster of an over-sized grid waits for a slot only to find that its unit does not exist.
-    static int32_t occ_smem = -1, occ_c = -1, occ_clusters = 0;
+    static int32_t occ_smem_d[DEVICE_TABLE] = {}, occ_c_d[DEVICE_TABLE] = {}, occ_clusters_d[DEVICE_TABLE] = {};
+    int32_t &occ_smem = occ_smem_d[dv], &occ_c = occ_c_d[dv], &occ_clusters = occ_clusters_d[dv];
     if (occ_smem != smem || occ_c != C) {
         cfg.gridDim = dim3((unsigned)(C * pool->sm_count), 1, 1);
         cfg.numAttrs = 1;

@@ -581,7 +581,8 @@ static lora_status_t launch_tc_bucket(lora_pool_t *pool, const TcParams &P, cons
         return LORA_ERR_INVALID_ARG;
 
     constexpr int SH_SMEM = SH_STAGES * (XT_BYTES + ((RP * 128 + 1023) & ~1023)) + 256 + 1024;
-    static bool attr_done = false;
+    static bool attr_done_d[DEVICE_TABLE] = {};
+    bool &attr_done = attr_done_d[device_index(pool->device)];
     if (!attr_done) {
         LORA_CUDA_TRY(cudaFuncSetAttribute(tc_shrink_kernel<RP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            SH_SMEM));

@@ -104,6 +104,11 @@ __host__ __device__ inline MetaLayout meta_layout(int32_t T, int32_t num_slots, 
     return L;
 }
 
+// Kernel attributes (dynamic shared-memory limits) and occupancy figures are per device: the
+// launchers keep what they have set or asked in small tables indexed by the device ordinal.
+constexpr int DEVICE_TABLE = 64;
+inline int device_index(int device) { return device >= 0 && device < DEVICE_TABLE ? device : 0; }
+
 // rank bucket a slot's kernels are specialised for: 8, 16, 32 or 64
 __host__ __device__ inline int32_t rank_bucket(int32_t r) {
     return r <= 8 ? 8 : r <= 16 ? 16 : r <= 32 ? 32 : 64;
