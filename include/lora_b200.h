@@ -26,7 +26,10 @@
  *    stream given; the library never synchronises a device and never allocates device memory;
  *  - bf16 tensors are row-major with a leading dimension in ELEMENTS; base pointers must be
  *    16-byte aligned and every d_in, d_out and leading dimension a multiple of 8;
- *  - arithmetic: bf16 inputs, fp32 accumulation, one round-to-nearest-even to bf16 at the store.
+ *  - arithmetic: bf16 inputs, fp32 accumulation, one round-to-nearest-even to bf16 at the store;
+ *  - a pool handle keeps host-side state (slot table copy, events, tensor maps, the shapes of the
+ *    metadata tables built through it) and is not thread-safe: calls on one pool come from one
+ *    host thread at a time.  Different pools are independent.
  */
 #ifndef LORA_B200_H
 #define LORA_B200_H
