@@ -155,6 +155,7 @@ lora_status_t lora_pool_reset_status(lora_pool_t *pool, void *stream);
  *   key 3  fused kernel: upper bound on the clusters in the grid
  *   key 4  tensor-core kernels of lora_sgmv_apply: 1 = never, 2 = whenever they apply
  *   key 5  fused kernel: stages of the shared-memory ring (2 .. 4)
+ *   key 6  fused kernel: 1 = partial sums always fetched from the cluster's blocks, never pushed
  *   key 7  segment builder: 1 = one warp per slot also for long batches
  * Keys outside 0 .. 7 -> INVALID_ARG. */
 lora_status_t lora_pool_set_tuning(lora_pool_t *pool, int32_t key, int32_t value);

@@ -55,6 +55,7 @@ void fill_apply_params(lora_pool_t *pool, ApplyParams &P, int32_t target, const 
     P.moff_perm = P.moff_udesc = P.moff_uperm = 0;
     P.path_filter = 0;
     P.early = 0;
+    P.push = 0;
 }
 
 static lora_status_t apply_common(lora_pool_t *pool, int32_t target, const void *x, int64_t ldx,

@@ -27,6 +27,7 @@ struct ApplyParams {
     int32_t off_part, off_vpart, off_vh, off_vl;   // warp partials, block partial, v as bf16 high / low parts
     int32_t off_stage, stage_bytes, n_stages;      // ring of job buffers
     int32_t moff_perm, moff_udesc, moff_uperm;     // word offsets: perm, unit records, unit row ids
+    int32_t push;              // fused path: block partials are pushed to all blocks of the cluster (small units)
     int32_t early;             // the unit records and the pool may be read before the preceding kernel has finished
     int32_t path_filter;       // 0 = every unit; else skip runs of at least this many consecutive tokens
 };

@@ -19,7 +19,9 @@
 //   shrink  partial v over the block's d_in slice, the four warps splitting rank tiles and columns,
 //           bf16 tensor-core MMA (m16n8k16) with fp32 accumulation carried across chunks in registers;
 //   exchange the block partials are summed through distributed shared memory in block order,
-//           identically in every block (no global workspace, no float atomics);
+//           identically in every block (no global workspace, no float atomics): small units push
+//           their partial into every block of the cluster and sum locally after one barrier,
+//           larger ones fetch the partials from the blocks that hold them;
 //   expand  over the block's d_out slice on the tensor cores, v carried as the sum of two bf16
 //           numbers (high and low part, ~16 mantissa bits); scale and residual add fused, y_base
 //           read from the job's stage, one rounding to bf16 at the store.
@@ -125,6 +127,12 @@ __device__ __forceinline__ float ld_peer_f32(uint32_t local_addr, uint32_t rank)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
     asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
     return v;
+}
+// write a float at the same shared-memory offset in block `rank` of the cluster
+__device__ __forceinline__ void st_peer_f32(uint32_t local_addr, uint32_t rank, float v) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
 }
 // D += A(16x16, row) . B(16x8, col), bf16 inputs, fp32 accumulate
 __device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
@@ -337,6 +345,7 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
     unsigned char *smem = cx.smem;
     float *part = reinterpret_cast<float *>(smem + P.off_part);     // [WK][mrows][RP] = mrows x 64 floats
     float *vpart = reinterpret_cast<float *>(smem + P.off_vpart);   // [mrows][RP], read by the peers
+    float *vall = vpart;   // push mode: [cluster size][mrows][RP], written by the peers
     __nv_bfloat16 *Vh = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_vh);   // [mrows][PV]
     __nv_bfloat16 *Vl = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_vl);
 
@@ -397,7 +406,14 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
             float v = part[i];
 #pragma unroll
             for (int w = 1; w < WK; ++w) v += part[w * mrows * RP + i];
-            vpart[i] = v;
+            if (P.push) {
+                // small units: every block hands its partial to all blocks (remote stores need no
+                // answer), so that after the barrier the sum is taken from local shared memory
+                const uint32_t dst = smem_u32(vall + ((int)cx.crank * mrows * RP + i));
+                for (uint32_t q = 0; q < cx.csize; ++q) st_peer_f32(dst, q, v);
+            } else {
+                vpart[i] = v;
+            }
         }
     }
     // ---- exchange: every block sums all blocks' partials in block order -------------------------
@@ -414,7 +430,9 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
                 float pv[8];
 #pragma unroll
                 for (uint32_t q = 0; q < 8; ++q)
-                    pv[q] = q < cx.csize ? ld_peer_f32(vp_addr + (uint32_t)(m * RP + k) * 4u, q) : 0.0f;
+                    pv[q] = q >= cx.csize ? 0.0f
+                            : P.push     ? vall[(int)q * mrows * RP + m * RP + k]
+                                         : ld_peer_f32(vp_addr + (uint32_t)(m * RP + k) * 4u, q);
 #pragma unroll
                 for (uint32_t q = 0; q < 8; ++q) v += pv[q];
             }
@@ -699,7 +717,10 @@ static lora_status_t launch_h(lora_pool_t *pool, ApplyParams P, int32_t C, const
     if (S < 2 || S > MAX_STAGES) S = 2;   // two stages and more resident blocks beat deeper rings
     int32_t o = SM_HEADER;
     P.off_part = o;   o += mrows * 64 * 4;
-    P.off_vpart = o;  o += mrows * RPmax * 4;
+    // the partials of all blocks of the cluster fit beside each other when units are small: then
+    // they are pushed to every block instead of fetched by every block
+    P.push = (8 * mrows * RPmax * 4 <= 4096 && pool->tuning[6] != 1) ? 1 : 0;
+    P.off_vpart = o;  o += (P.push ? 8 : 1) * mrows * RPmax * 4;
     P.off_vh = o;     o += mrows * (RPmax + 8) * 2;
     P.off_vl = o;     o += mrows * (RPmax + 8) * 2;
     o = (o + 1023) & ~1023;
