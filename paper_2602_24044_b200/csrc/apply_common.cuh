@@ -116,13 +116,13 @@ __device__ __forceinline__ Tile resolve_unit(const ApplyParams &P, const MetaLay
 // y_base -> y for rows that take no adapter (out-of-place calls only); the columns are split
 // over `parts` blocks, this block being number `part`.
 __device__ __forceinline__ void copy_rows(const ApplyParams &P, const int32_t *rowidx, int32_t rows,
-                                          int32_t part, int32_t parts) {
+                                          int32_t part, int32_t parts, int32_t nthreads = 0) {
+    if (nthreads == 0) nthreads = (int32_t)blockDim.x;   // threads that take part (the first ones of the block)
     const int32_t vecs = P.tv.d_out / 8;
     for (int32_t m = 0; m < rows; ++m) {
         const __nv_bfloat16 *src = P.yb + (int64_t)rowidx[m] * P.ldyb;
         __nv_bfloat16 *dst = P.y + (int64_t)rowidx[m] * P.ldy;
-        for (int32_t v = part * (int32_t)blockDim.x + threadIdx.x; v < vecs;
-             v += parts * (int32_t)blockDim.x)
+        for (int32_t v = part * nthreads + threadIdx.x; v < vecs; v += parts * nthreads)
             reinterpret_cast<uint4 *>(dst)[v] = ldg16(src + (int64_t)v * 8);
     }
 }

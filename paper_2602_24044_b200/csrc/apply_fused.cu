@@ -34,7 +34,8 @@
 
 namespace lora {
 
-constexpr int FT = 128;          // threads per block
+constexpr int FT = 128;          // consumer threads per block (four warps)
+constexpr int FT_ALL = 160;      // plus the warp that requests the jobs
 constexpr int UNIT_RING = 4;     // unit records held in shared memory: previous, current, next, next but one
 constexpr int RING_ENTRY = 80;   // one record: 16 bytes + 16 row ids
 constexpr int SM_RING = 64;      // byte offset of the record ring (mbarriers come first)
@@ -70,6 +71,11 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
                  "r"(bytes)
                  : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// barrier among the four consumer warps (the requesting warp runs on its own)
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -251,85 +257,124 @@ __device__ __forceinline__ void store_unit(unsigned char *smem, int32_t iter, co
 struct Ctx {
     unsigned char *smem;
     uint64_t *full;            // [n_stages] a job's data has landed
+    uint64_t *empty;           // [n_stages] the four consumer warps are done with the stage
     int32_t cid, G, n_units;   // cluster index, clusters in the grid, units in the batch
     uint32_t crank, csize;
     int32_t a_lo, a_hi, b_lo, b_hi;   // this block's column slices of d_in and d_out
     int32_t ci;                // unit iteration the consumers work on
     int32_t cq;                // jobs consumed so far
-    int32_t pi, pj, pq;        // producer: unit iteration, job within it, jobs requested so far
     bool pending_wait;         // a cluster barrier arrive whose wait is still to come
     bool ok;                   // no wait has expired
 };
 
-// Position in the block's job stream -> the job's unit and row ids.  Moves (it_i, it_j) past
-// units without jobs.  False when the stream has no further job that may be requested yet: jobs of
-// the unit after the current one may be (their record is in the ring), anything further waits.
-__device__ __forceinline__ bool peek_job(const ApplyParams &P, const Ctx &cx, int32_t &it_i, int32_t &it_j,
-                                         Unit &un, const int32_t *&rowidx) {
-    for (;;) {
-        if (it_i > cx.ci + 1 || cx.cid + it_i * cx.G >= cx.n_units) return false;
-        const unsigned char *e = cx.smem + SM_RING + (it_i % UNIT_RING) * RING_ENTRY;
-        un = decode_unit(P, *reinterpret_cast<const int4 *>(e), cx.a_hi - cx.a_lo, cx.b_hi - cx.b_lo);
-        rowidx = reinterpret_cast<const int32_t *>(e + 16);
-        if (un.run && it_j < un.na + un.nb) return true;
-        ++it_i;
-        it_j = 0;
+// Requesting warp: one job into stage `st`.  mode 0: whole job; 1: only the weight tile (and the
+// byte count of the whole job); 2: only the token rows of a job whose tile was requested in mode 1.
+// Lane l < 16 holds the id of the unit's row l in `rowid`.
+__device__ __forceinline__ void request_job(const ApplyParams &P, const FusedMaps &M, const Ctx &cx,
+                                            const Unit &un, int32_t j, int st, int32_t rowid, int lane,
+                                            int mode) {
+    unsigned char *ws = cx.smem + P.off_stage + st * P.stage_bytes;
+    const bool shrink = j < un.na;
+    const int32_t c = shrink ? j : j - un.na;
+    const int32_t col0 = (shrink ? cx.a_lo : cx.b_lo) + c * un.CW;   // a multiple of 64
+    const int32_t ncols = min(un.CW, (shrink ? cx.a_hi : cx.b_hi) - col0);
+    const int32_t pitch = un.CW + 8;
+    const CUtensorMap *map = shrink ? &M.a[(un.rb >> 3) - 1] : &M.b[(un.rb >> 3) - 1];
+    const __nv_bfloat16 *tok = (shrink ? P.x : P.yb) + col0;
+    const int64_t tld = shrink ? P.ldx : P.ldyb;
+    __nv_bfloat16 *ts = reinterpret_cast<__nv_bfloat16 *>(ws + W_BYTES);
+    if (lane == 0 && mode != 2) {
+        // the tile load always delivers its whole box: rb rows of CW columns
+        mbar_expect_tx(&cx.full[st], (uint32_t)un.rb * (uint32_t)un.CW * 2u +
+                                         (uint32_t)un.rows * (uint32_t)ncols * 2u);
+        tma_load_4d(ws, map, 0, 0, col0 >> 6, un.slot, &cx.full[st]);
     }
+    __syncwarp();
+    if (lane < un.rows && mode != 1)
+        bulk_g2s(ts + lane * pitch, tok + (int64_t)rowid * tld, (uint32_t)ncols * 2u, &cx.full[st]);
 }
 
-// Warp 0: request jobs until the ring is full.
-// mode 0: whole jobs; 1: only the weight tiles (and the byte count of the whole job); 2: only the
-// token rows of jobs whose weight tiles were requested in mode 1 (same walk, from the same state).
-__device__ __forceinline__ void issue_jobs(const ApplyParams &P, const FusedMaps &M, Ctx &cx, int lane,
-                                           int mode = 0) {
+// The requesting warp: walks the same units as the consumers (it reads the records itself, one
+// unit ahead, into registers), and keeps the ring full: a job is requested as soon as the four
+// consumer warps have left its stage, whatever they are doing meanwhile, so the time it takes to
+// issue copies is off their critical path.  It takes part in the cluster barriers of every unit
+// (all threads of a cluster count there), after the unit's last job has been requested.
+__device__ __forceinline__ void producer_warp(const ApplyParams &P, const FusedMaps &M, Ctx &cx, int lane) {
     const int32_t S = P.n_stages;
-    Unit un;
-    const int32_t *rowidx;
-    while (cx.pq - cx.cq < S && peek_job(P, cx, cx.pi, cx.pj, un, rowidx)) {
-        const int st = cx.pq % S;
-        unsigned char *ws = cx.smem + P.off_stage + st * P.stage_bytes;
-        const bool shrink = cx.pj < un.na;
-        const int32_t c = shrink ? cx.pj : cx.pj - un.na;
-        const int32_t col0 = (shrink ? cx.a_lo : cx.b_lo) + c * un.CW;   // a multiple of 64
-        const int32_t ncols = min(un.CW, (shrink ? cx.a_hi : cx.b_hi) - col0);
-        const int32_t pitch = un.CW + 8;
-        const CUtensorMap *map = shrink ? &M.a[(un.rb >> 3) - 1] : &M.b[(un.rb >> 3) - 1];
-        const __nv_bfloat16 *tok = (shrink ? P.x : P.yb) + col0;
-        const int64_t tld = shrink ? P.ldx : P.ldyb;
-        __nv_bfloat16 *ts = reinterpret_cast<__nv_bfloat16 *>(ws + W_BYTES);
-        if (lane == 0 && mode != 2) {
-            // the tile load always delivers its whole box: rb rows of CW columns
-            mbar_expect_tx(&cx.full[st], (uint32_t)un.rb * (uint32_t)un.CW * 2u +
-                                             (uint32_t)un.rows * (uint32_t)ncols * 2u);
-            tma_load_4d(ws, map, 0, 0, col0 >> 6, un.slot, &cx.full[st]);
+    int32_t n_units = P.meta ? ldg_int(P.meta + H_NPIECE) : P.T;
+    UnitRegs cur = fetch_unit(P, cx.cid, P.units, lane);
+    if (n_units > P.units) n_units = P.units;
+    int32_t q = 0, skip = 0;
+    bool pending = false, ok = true;
+    for (int32_t i = 0;; ++i) {
+        const int32_t u = cx.cid + i * cx.G;
+        if (u >= n_units) {
+            if (i == 0 && P.early) griddep_wait();
+            break;
         }
-        __syncwarp();
-        if (lane < un.rows && mode != 1)
-            bulk_g2s(ts + lane * pitch, tok + (int64_t)rowidx[lane] * tld, (uint32_t)ncols * 2u,
-                     &cx.full[st]);
-        ++cx.pj;
-        ++cx.pq;
+        const UnitRegs nxt = fetch_unit(P, u + cx.G, n_units, lane);   // the next unit's record, meanwhile
+        int4 rec;
+        rec.x = __shfl_sync(0xffffffffu, cur.rec.x, 16);
+        rec.y = __shfl_sync(0xffffffffu, cur.rec.y, 16);
+        rec.z = __shfl_sync(0xffffffffu, cur.rec.z, 16);
+        rec.w = __shfl_sync(0xffffffffu, cur.rec.w, 16);
+        const Unit un = decode_unit(P, rec, cx.a_hi - cx.a_lo, cx.b_hi - cx.b_lo);
+        const int32_t njobs = un.run ? un.na + un.nb : 0;
+        if (i == 0 && P.early) {
+            // The kernel before this one may still be running: the pool may be read (the host
+            // vouches for it), the activations not yet.  Weight tiles of the first jobs now, their
+            // token rows after the wait.
+            skip = njobs < S ? njobs : S;
+            for (int32_t j = 0; j < skip; ++j) request_job(P, M, cx, un, j, j, cur.rowid, lane, 1);
+            griddep_wait();
+            for (int32_t j = 0; j < skip; ++j) request_job(P, M, cx, un, j, j, cur.rowid, lane, 2);
+        }
+        // The unit's two cluster barriers are taken in step with the consumers, who pass the first
+        // one between the shrink and the expand jobs: arrive there BEFORE requesting expand jobs
+        // (their stages only come free once the consumers are past it), wait for it afterwards.
+        const int32_t n_shrink = un.run ? un.na : 0;
+        for (int32_t j = 0; j < njobs; ++j, ++q) {
+            if (j == n_shrink && un.run) {
+                if (pending) cluster_wait();
+                cluster_arrive();
+            }
+            if (i == 0 && j < skip) continue;
+            const int st = q % S;
+            if (q >= S) ok = mbar_wait(&cx.empty[st], (uint32_t)(q / S - 1) & 1u) && ok;
+            request_job(P, M, cx, un, j, st, cur.rowid, lane, 0);
+        }
+        if (un.run) {
+            if (njobs == n_shrink) {   // no expand job in this block: the first barrier is still to come
+                if (pending) cluster_wait();
+                cluster_arrive();
+            }
+            cluster_wait();
+            cluster_arrive();
+            pending = true;
+        }
+        cur = nxt;
     }
+    if (pending) cluster_wait();
+    if (!ok && lane == 0) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
 }
 
-// All threads: wait for the data of the next job; returns its stage.
+// Consumers: wait for the data of the next job; returns its stage.
 __device__ __forceinline__ const unsigned char *acquire_job(const ApplyParams &P, Ctx &cx) {
     const int st = cx.cq % P.n_stages;
     cx.ok = mbar_wait(&cx.full[st], (uint32_t)(cx.cq / P.n_stages) & 1u) && cx.ok;
     return cx.smem + P.off_stage + st * P.stage_bytes;
 }
-// All threads: the job's stage is free again; warp 0 refills the ring.
-__device__ __forceinline__ void release_job(const ApplyParams &P, const FusedMaps &M, Ctx &cx, int warp,
-                                            int lane) {
-    __syncthreads();
+// Consumers: this warp is done with the job's stage.
+__device__ __forceinline__ void release_job(const ApplyParams &P, Ctx &cx, int lane) {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&cx.empty[cx.cq % P.n_stages]);
     ++cx.cq;
-    if (warp == 0) issue_jobs(P, M, cx, lane);
 }
 
 // RP: rank bucket of the unit; H: 1 when a unit holds at most 8 rows, 2 when rows 8..15 can be occupied.
 template <int RP, int H>
-__device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps &M, const Unit &un,
-                                          const int32_t *rowidx, Ctx &cx) {
+__device__ __forceinline__ void unit_body(const ApplyParams &P, const Unit &un, const int32_t *rowidx,
+                                          Ctx &cx) {
     constexpr int CW = 4096 / RP;      // columns per job
     constexpr int PW = CW + 8;         // row pitch of the token rows: +16 B against bank conflicts
     constexpr int PV = RP + 8;         // pitch of the bf16 copies of v
@@ -385,7 +430,7 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
                 }
             }
         }
-        release_job(P, M, cx, warp, lane);
+        release_job(P, cx, lane);
     }
     // the peers have finished reading the previous unit's partial before it is overwritten
     if (cx.pending_wait) {
@@ -398,7 +443,7 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
         *reinterpret_cast<float2 *>(p0) = make_float2(acc[i][0], acc[i][1]);
         if (hi_rows) *reinterpret_cast<float2 *>(p0 + 8 * RP) = make_float2(acc[i][2], acc[i][3]);
     }
-    __syncthreads();
+    consumer_sync();
     // block partial: the column splits' sums in order
     for (int i = tid; i < mrows * RP; i += FT) {
         const int r = i / RP;
@@ -443,7 +488,7 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
     }
     cluster_arrive();   // done reading the peers; the matching wait comes before the next overwrite
     cx.pending_wait = true;
-    __syncthreads();
+    consumer_sync();
 
     // ---- expand: warp w takes columns [w*NW, (w+1)*NW) of every chunk ---------------------------
     const float s = un.scale;
@@ -509,13 +554,13 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const FusedMaps 
                 }
             }
         }
-        release_job(P, M, cx, warp, lane);
+        release_job(P, cx, lane);
     }
 }
 
 // H: 1 when a unit holds at most 8 rows (decode tiles, single tokens), 2 otherwise.
 template <int H>
-__global__ void __launch_bounds__(FT, LORA_FUSED_MIN_BLOCKS)
+__global__ void __launch_bounds__(FT_ALL, LORA_FUSED_MIN_BLOCKS)
 fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
     extern __shared__ __align__(1024) unsigned char smem[];
     Ctx cx;
@@ -533,8 +578,12 @@ fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
     }
 
     // barriers; the next lines touch no memory another kernel writes
+    cx.empty = cx.full + MAX_STAGES;
     if (tid == 0) {
-        for (int s = 0; s < P.n_stages; ++s) mbar_init(&cx.full[s], 1);
+        for (int s = 0; s < P.n_stages; ++s) {
+            mbar_init(&cx.full[s], 1);
+            mbar_init(&cx.empty[s], 4);
+        }
         fence_mbar_init();
     }
     // this block's column slices (multiples of 64 columns: tile loads address whole column blocks)
@@ -546,16 +595,24 @@ fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
         cx.b_lo = min((int32_t)cx.crank * Wb, P.tv.d_out);
         cx.b_hi = min(cx.b_lo + Wb, P.tv.d_out);
     }
+    // zeros in every stage (rows above a unit's rank are never copied, and what they hold is
+    // multiplied by zeros of v, so it has to be finite)
+    for (int i = tid; i < P.n_stages * P.stage_bytes / 16; i += FT_ALL)
+        reinterpret_cast<uint4 *>(smem + P.off_stage)[i] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async();   // the stages are written by bulk copies from here on
     // Under programmatic dependent launch this kernel may start while the one before it on the
     // stream is still running.  Activations are only touched after griddep_wait().  The unit
     // records and the pool were complete before that kernel started when P.early is set (the host
     // sets it only then), so they are read, and the first weight tiles requested, ahead of the wait.
-    if (!P.early) {
-        // nothing may be read yet: use the time for the zeros in every stage (rows above a unit's
-        // rank are never copied, and what they hold is multiplied by zeros of v, so it has to be finite)
-        for (int i = tid; i < P.n_stages * P.stage_bytes / 16; i += FT)
-            reinterpret_cast<uint4 *>(smem + P.off_stage)[i] = make_uint4(0, 0, 0, 0);
-        griddep_wait();
+    if (!P.early) griddep_wait();
+    __syncthreads();
+    cx.ci = 0;
+    cx.cq = 0;
+    cx.pending_wait = false;
+    cx.ok = true;
+    if (warp == 4) {   // the requesting warp goes its own way from here
+        producer_warp(P, M, cx, lane);
+        return;
     }
     {
         // the number of units and the records of this cluster's first two units, side by side
@@ -565,30 +622,14 @@ fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
             m1 = fetch_unit(P, cx.cid + cx.G, P.units, lane);
         }
         cx.n_units = P.meta ? ldg_int(P.meta + H_NPIECE) : P.T;
-        // meanwhile (early mode): the zeros in every stage
-        if (P.early)
-            for (int i = tid; i < P.n_stages * P.stage_bytes / 16; i += FT)
-                reinterpret_cast<uint4 *>(smem + P.off_stage)[i] = make_uint4(0, 0, 0, 0);
-        fence_proxy_async();   // the stages are written by bulk copies from here on
         if (cx.n_units > P.units) cx.n_units = P.units;
         if (warp == 3) {
             store_unit(smem, 0, m0, cx.cid < cx.n_units, lane);
             store_unit(smem, 1, m1, cx.cid + cx.G < cx.n_units, lane);
         }
     }
-    __syncthreads();
-    cx.ci = 0;
-    cx.cq = cx.pq = cx.pi = cx.pj = 0;
-    cx.pending_wait = false;
-    cx.ok = true;
-    if (P.early) {
-        if (warp == 0) issue_jobs(P, M, cx, lane, 1);
-        griddep_wait();
-        if (warp == 0) {
-            cx.pi = cx.pj = cx.pq = 0;
-            issue_jobs(P, M, cx, lane, 2);
-        }
-    }
+    consumer_sync();
+    if (P.early) griddep_wait();
     // the next kernel on the stream may be scheduled from here on: everything older than this
     // kernel is complete
     griddep_launch_dependents();
@@ -603,17 +644,16 @@ fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
         const int4 rec = *reinterpret_cast<const int4 *>(e);
         const int32_t *rowidx = reinterpret_cast<const int32_t *>(e + 16);
         const Unit un = decode_unit(P, rec, cx.a_hi - cx.a_lo, cx.b_hi - cx.b_lo);
-        if (warp == 0) issue_jobs(P, M, cx, lane);
         if (un.run) {
-            if (un.RP == 16) unit_body<16, H>(P, M, un, rowidx, cx);
-            else if (un.RP == 32) unit_body<32, H>(P, M, un, rowidx, cx);
-            else unit_body<64, H>(P, M, un, rowidx, cx);
+            if (un.RP == 16) unit_body<16, H>(P, un, rowidx, cx);
+            else if (un.RP == 32) unit_body<32, H>(P, un, rowidx, cx);
+            else unit_body<64, H>(P, un, rowidx, cx);
         } else if (!P.meta && rec.x == -1) {   // per-token mode: this token has no adapter
             if (cx.crank == 0 && tid == 0 && rec.y) atomicAdd(&P.pool.status[STATUS_INVALID_TOKENS], 1);
-            if (!P.in_place) copy_rows(P, rowidx, 1, (int32_t)cx.crank, (int32_t)cx.csize);
+            if (!P.in_place) copy_rows(P, rowidx, 1, (int32_t)cx.crank, (int32_t)cx.csize, FT);
         }
         if (warp == 3) store_unit(smem, cx.ci + 2, mn, true, lane);
-        __syncthreads();   // the new record is visible; nobody reads the current one any more
+        consumer_sync();   // the new record is visible; nobody reads the current one any more
     }
     if (!cx.ok && tid == 0) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
 
@@ -623,10 +663,10 @@ fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
         const int32_t n_active = __ldg(P.meta + H_NACTIVE);
         for (int32_t first = cx.cid * 16; first < P.T - n_active; first += cx.G * 16) {
             const int32_t rows = min(16, P.T - n_active - first);
-            __syncthreads();
+            consumer_sync();
             if (tid < rows) rowidx[tid] = __ldg(P.meta + P.moff_perm + n_active + first + tid);
-            __syncthreads();
-            copy_rows(P, rowidx, rows, (int32_t)cx.crank, (int32_t)cx.csize);
+            consumer_sync();
+            copy_rows(P, rowidx, rows, (int32_t)cx.crank, (int32_t)cx.csize, FT);
         }
     }
     // no block leaves while a peer may still read its partials
@@ -736,7 +776,7 @@ static lora_status_t launch_h(lora_pool_t *pool, ApplyParams P, int32_t C, const
         attr_smem[dv] = smem;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.blockDim = dim3(FT, 1, 1);
+    cfg.blockDim = dim3(FT_ALL, 1, 1);
     cfg.dynamicSmemBytes = (size_t)smem;
     cfg.stream = stream;
     cudaLaunchAttribute at[2];
