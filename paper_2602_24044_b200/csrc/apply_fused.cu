@@ -10,8 +10,11 @@
 // (TMA, 128-byte swizzle, the matrix viewed as blocks of 64 columns), plus the unit's rows of x (or
 // y_base), one bulk copy per row, into one stage of a small ring of shared-memory buffers
 // (mbarrier-signalled).  Few large copies matter: every bulk copy costs the issuing thread and the
-// copy engine a fixed time, and a copy per weight row made that time the bottleneck.  Warp 0 keeps
-// the ring full: whenever a stage has been consumed it requests the next job of the stream, which may belong to the next unit, so the memory latency of
+// copy engine a fixed time, and a copy per weight row made that time the bottleneck.  A fifth
+// warp does nothing but request jobs: it reads the unit records itself, one unit ahead, and refills
+// a stage as soon as the four consumer warps have left it (per-stage mbarriers), so issuing copies
+// (0.4-0.7 us per job when a consumer warp did it) is off the consumers' critical path, and the
+// next job of the stream may belong to the next unit, so the memory latency of
 // a unit hides behind the arithmetic of the one before.  The chunk width shrinks as the rank
 // grows (256 / 128 / 64 columns for ranks <= 16 / 32 / 64), so a stage is the same size for
 // every rank and one launch serves all of them.
