@@ -23,8 +23,9 @@
 //           bf16 tensor-core MMA (m16n8k16) with fp32 accumulation carried across chunks in registers;
 //   exchange the block partials are summed through distributed shared memory in block order,
 //           identically in every block (no global workspace, no float atomics): small units push
-//           their partial into every block of the cluster and sum locally after one barrier,
-//           larger ones fetch the partials from the blocks that hold them;
+//           their partial into every block of the cluster and sum locally, larger ones fetch the
+//           partials from the blocks that hold them; the blocks signal each other through
+//           mbarriers in each other's shared memory (bounded waits), not the hardware cluster barrier;
 //   expand  over the block's d_out slice on the tensor cores, v carried as the sum of two bf16
 //           numbers (high and low part, ~16 mantissa bits); scale and residual add fused, y_base
 //           read from the job's stage, one rounding to bf16 at the store.
@@ -42,7 +43,9 @@ constexpr int FT_ALL = 160;      // plus the warp that requests the jobs
 constexpr int UNIT_RING = 4;     // unit records held in shared memory: previous, current, next, next but one
 constexpr int RING_ENTRY = 80;   // one record: 16 bytes + 16 row ids
 constexpr int SM_RING = 64;      // byte offset of the record ring (mbarriers come first)
-constexpr int SM_HEADER = 384;   // bytes before the first carved-up buffer
+constexpr int SM_XBAR = 384;     // mbarrier: every block of the cluster has published its partial
+constexpr int SM_YBAR = 392;     // mbarrier: every block of the cluster has read the partials
+constexpr int SM_HEADER = 448;   // bytes before the first carved-up buffer
 constexpr int MAX_STAGES = 4;
 constexpr int W_BYTES = 8192;    // weight tile of a job: rank bucket x chunk width x 2 bytes, for every bucket
 
@@ -128,6 +131,28 @@ __device__ __forceinline__ void cluster_arrive() {
 }
 __device__ __forceinline__ void cluster_wait() {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// one arrival on the mbarrier at the same shared-memory offset in block `rank` of the cluster; the
+// arriving thread's earlier writes and reads are ordered before it (release at cluster scope)
+__device__ __forceinline__ void mbar_arrive_peer(uint64_t *local_bar, uint32_t rank) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local_bar)), "r"(rank));
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+// bounded wait on this block's mbarrier for arrivals from the whole cluster (acquire at cluster scope)
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity) {
+    for (uint32_t i = 0; i < (1u << 20); ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
 }
 // read a float at the same shared-memory offset in block `rank` of the cluster
 __device__ __forceinline__ float ld_peer_f32(uint32_t local_addr, uint32_t rank) {
@@ -266,7 +291,7 @@ struct Ctx {
     int32_t a_lo, a_hi, b_lo, b_hi;   // this block's column slices of d_in and d_out
     int32_t ci;                // unit iteration the consumers work on
     int32_t cq;                // jobs consumed so far
-    bool pending_wait;         // a cluster barrier arrive whose wait is still to come
+    int32_t k_run;             // units this block has exchanged partials for (phase of the two mbarriers)
     bool ok;                   // no wait has expired
 };
 
@@ -300,15 +325,14 @@ __device__ __forceinline__ void request_job(const ApplyParams &P, const FusedMap
 // The requesting warp: walks the same units as the consumers (it reads the records itself, one
 // unit ahead, into registers), and keeps the ring full: a job is requested as soon as the four
 // consumer warps have left its stage, whatever they are doing meanwhile, so the time it takes to
-// issue copies is off their critical path.  It takes part in the cluster barriers of every unit
-// (all threads of a cluster count there), after the unit's last job has been requested.
+// issue copies is off their critical path.
 __device__ __forceinline__ void producer_warp(const ApplyParams &P, const FusedMaps &M, Ctx &cx, int lane) {
     const int32_t S = P.n_stages;
     int32_t n_units = P.meta ? ldg_int(P.meta + H_NPIECE) : P.T;
     UnitRegs cur = fetch_unit(P, cx.cid, P.units, lane);
     if (n_units > P.units) n_units = P.units;
     int32_t q = 0, skip = 0;
-    bool pending = false, ok = true;
+    bool ok = true;
     for (int32_t i = 0;; ++i) {
         const int32_t u = cx.cid + i * cx.G;
         if (u >= n_units) {
@@ -332,32 +356,14 @@ __device__ __forceinline__ void producer_warp(const ApplyParams &P, const FusedM
             griddep_wait();
             for (int32_t j = 0; j < skip; ++j) request_job(P, M, cx, un, j, j, cur.rowid, lane, 2);
         }
-        // The unit's two cluster barriers are taken in step with the consumers, who pass the first
-        // one between the shrink and the expand jobs: arrive there BEFORE requesting expand jobs
-        // (their stages only come free once the consumers are past it), wait for it afterwards.
-        const int32_t n_shrink = un.run ? un.na : 0;
         for (int32_t j = 0; j < njobs; ++j, ++q) {
-            if (j == n_shrink && un.run) {
-                if (pending) cluster_wait();
-                cluster_arrive();
-            }
             if (i == 0 && j < skip) continue;
             const int st = q % S;
             if (q >= S) ok = mbar_wait(&cx.empty[st], (uint32_t)(q / S - 1) & 1u) && ok;
             request_job(P, M, cx, un, j, st, cur.rowid, lane, 0);
         }
-        if (un.run) {
-            if (njobs == n_shrink) {   // no expand job in this block: the first barrier is still to come
-                if (pending) cluster_wait();
-                cluster_arrive();
-            }
-            cluster_wait();
-            cluster_arrive();
-            pending = true;
-        }
         cur = nxt;
     }
-    if (pending) cluster_wait();
     if (!ok && lane == 0) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
 }
 
@@ -435,11 +441,13 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const Unit &un, 
         }
         release_job(P, cx, lane);
     }
-    // the peers have finished reading the previous unit's partial before it is overwritten
-    if (cx.pending_wait) {
-        cluster_wait();
-        cx.pending_wait = false;
-    }
+    // The exchange is signalled with two mbarriers per block instead of the cluster-wide hardware
+    // barrier (0.8 us a round even without skew): every block of the cluster arrives on every block's
+    // barrier, once when its partial is published, once when it has read the partials.
+    uint64_t *xbar = reinterpret_cast<uint64_t *>(smem + SM_XBAR);
+    uint64_t *ybar = reinterpret_cast<uint64_t *>(smem + SM_YBAR);
+    // the peers have finished reading the previous unit's partials before they are overwritten
+    if (cx.k_run > 0) cx.ok = mbar_wait_cluster(ybar, (uint32_t)(cx.k_run - 1) & 1u) && cx.ok;
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
         float *p0 = part + (wk * mrows + g) * RP + (wn * 2 + i) * 8 + 2 * t;
@@ -465,8 +473,11 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const Unit &un, 
         }
     }
     // ---- exchange: every block sums all blocks' partials in block order -------------------------
-    cluster_arrive();
-    cluster_wait();
+    // one arrival per block and peer: thread q tells block q, after the block's threads have met
+    // (its release then covers all their writes)
+    consumer_sync();
+    if (tid < (int)cx.csize) mbar_arrive_peer(xbar, (uint32_t)tid);
+    cx.ok = mbar_wait_cluster(xbar, (uint32_t)cx.k_run & 1u) && cx.ok;
     {
         const uint32_t vp_addr = smem_u32(vpart);
         for (int i = tid; i < rows * rank16; i += FT) {
@@ -489,9 +500,10 @@ __device__ __forceinline__ void unit_body(const ApplyParams &P, const Unit &un, 
             Vl[m * PV + k] = __float2bfloat16_rn(v - __bfloat162float(hi));
         }
     }
-    cluster_arrive();   // done reading the peers; the matching wait comes before the next overwrite
-    cx.pending_wait = true;
+    ++cx.k_run;
     consumer_sync();
+    // done reading the partials; the matching wait comes before the next overwrite (or the exit)
+    if (tid < (int)cx.csize) mbar_arrive_peer(ybar, (uint32_t)tid);
 
     // ---- expand: warp w takes columns [w*NW, (w+1)*NW) of every chunk ---------------------------
     const float s = un.scale;
@@ -587,8 +599,12 @@ fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
             mbar_init(&cx.full[s], 1);
             mbar_init(&cx.empty[s], 4);
         }
+        mbar_init(reinterpret_cast<uint64_t *>(smem + SM_XBAR), cx.csize);
+        mbar_init(reinterpret_cast<uint64_t *>(smem + SM_YBAR), cx.csize);
         fence_mbar_init();
     }
+    // the only cluster-wide hardware barrier: no block signals a peer whose barriers are not set up
+    cluster_arrive();
     // this block's column slices (multiples of 64 columns: tile loads address whole column blocks)
     {
         const int32_t cs64 = (int32_t)cx.csize * 64;
@@ -609,9 +625,10 @@ fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
     // sets it only then), so they are read, and the first weight tiles requested, ahead of the wait.
     if (!P.early) griddep_wait();
     __syncthreads();
+    cluster_wait();
     cx.ci = 0;
     cx.cq = 0;
-    cx.pending_wait = false;
+    cx.k_run = 0;
     cx.ok = true;
     if (warp == 4) {   // the requesting warp goes its own way from here
         producer_warp(P, M, cx, lane);
@@ -672,8 +689,10 @@ fused_kernel(const ApplyParams P, const __grid_constant__ FusedMaps M) {
             copy_rows(P, rowidx, rows, (int32_t)cx.crank, (int32_t)cx.csize, FT);
         }
     }
-    // no block leaves while a peer may still read its partials
-    if (cx.pending_wait) cluster_wait();
+    // no block leaves while a peer may still read its partials or signal its barriers
+    if (cx.k_run > 0 && !mbar_wait_cluster(reinterpret_cast<uint64_t *>(smem + SM_YBAR),
+                                           (uint32_t)(cx.k_run - 1) & 1u) && tid == 0)
+        atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
 }
 
 // ---------------------------------------------------------------------------------------------
