@@ -208,8 +208,7 @@ def run_reference(args):
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "steps_timed": t["reps"], "ms_per_step": t["ms_per_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "config1 decode BGMV: 256 tokens, 4096->4096, 128 adapters "
-                                   "rank 16, Zipf(1.1)"},
+            "config": {"workload": workload_text(1, wl)},
             "cpu_baseline": {k: t[k] for k in ("value", "unit", "cores", "kind", "sample")},
             "e2e": {"value": t["value"], "unit": UNIT, "h2d_bytes_per_step": 0,
                     "d2h_bytes_per_step": 0},
@@ -227,6 +226,11 @@ WORKLOAD_TEXT = {
     4: "config4 full 32-layer decode step, Llama-3-8B shapes, LoRA on all 7 projections, 256 tokens, "
        "256 adapters rank 16, Zipf(1.1)",
 }
+
+
+def workload_text(cfg, wl):
+    """The `config.workload` string of a configuration: the same for both arms of the benchmark."""
+    return WORKLOAD_TEXT[cfg] + " (%d tokens, %d distinct adapters)" % (wl.T, len(wl.distinct_slots()))
 
 
 def case_workload(cfg):
@@ -353,65 +357,77 @@ def main():
     g_apply = capture(apply_only)
     torch.cuda.synchronize()
 
-    def run_steps(K, graph, fn):
-        with torch.cuda.stream(s.compute):
-            for _ in range(K // n_sets):
-                graph.replay()
-            for i in range(K % n_sets):
-                fn(i)
+    MIN_REGION_MS = 200.0      # every timed region lasts at least this long
 
-    K = args.steps if args.steps is not None else {0: 48000, 1: 48000, 2: 300, 3: 3000, 4: 100}[cfg]
+    def all_ranks_max_int(v):
+        return int(round(max_over_ranks(v, dev)))
+
+    def time_graph(graph, min_replays):
+        """Milliseconds for `n` back-to-back replays of a captured graph on the compute stream, with
+        n >= min_replays chosen so that the region lasts at least MIN_REGION_MS.  The graph is
+        replayed three times untimed first; nothing but whole replays runs inside the region."""
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(s.compute):
+            for _ in range(3):
+                graph.replay()
+            a.record(s.compute)
+            graph.replay()
+            b.record(s.compute)
+        torch.cuda.synchronize()
+        one = max(a.elapsed_time(b), 1e-4)
+        n = all_ranks_max_int(max(min_replays, int(np.ceil(MIN_REGION_MS / one))))
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(s.compute):
+            a.record(s.compute)
+            for _ in range(n):
+                graph.replay()
+            b.record(s.compute)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        return max_over_ranks(a.elapsed_time(b), dev), n
+
+    def run_steps(K, graph, fn):
+        """K steps as whole replays (K rounded up to a multiple of the graph's step count)."""
+        with torch.cuda.stream(s.compute):
+            for _ in range((K + n_sets - 1) // n_sets):
+                graph.replay()
+
+    K_req = args.steps if args.steps is not None else {0: 48000, 1: 48000, 2: 300, 3: 3000, 4: 100}[cfg]
     W_ = max(args.warmup, 3)
-    run_steps(min(W_, max(3, K // 4)), g_step, step)
+    run_steps(W_, g_step, step)
     torch.cuda.synchronize()
+    lb.pool_reset_status(s.pool, s.compute)
 
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    l0 = lb.launch_count()
-    e0.record(s.compute)
-    run_steps(K, g_step, step)
-    e1.record(s.compute)
-    torch.cuda.synchronize()
-    launches = (K // n_sets) * launches_per_rotation + (lb.launch_count() - l0)
-    if world > 1:
-        dist.barrier()
-    ms = max_over_ranks(e0.elapsed_time(e1), dev)
+    ms, n_rep = time_graph(g_step, (K_req + n_sets - 1) // n_sets)
+    K = n_rep * n_sets
+    launches = n_rep * launches_per_rotation
 
     # the applies alone (dominant kernel), same rotation, for the roofline figure
-    Kr = max(n_sets, min(K, 16000) // n_sets * n_sets)
-    r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    r0.record(s.compute)
-    run_steps(Kr, g_apply, apply_only)
-    r1.record(s.compute)
-    torch.cuda.synchronize()
     calls_per_step = len(sets[0])
-    apply_ms = r0.elapsed_time(r1) / Kr / calls_per_step
+    apply_total_ms, n_apply_rep = time_graph(g_apply, 1)
+    apply_ms = apply_total_ms / (n_apply_rep * n_sets) / calls_per_step
     # the same applies with ONE input / weight set replayed (small configurations: everything stays
     # in L2), reported beside the cold figure and labelled as warm
     warm_us = None
-    if n_sets > 1 and rank == 0:
+    if n_sets > 1:
         gw = torch.cuda.CUDAGraph()
         with torch.cuda.graph(gw, stream=s.compute):
             for _ in range(n_sets):
                 apply_calls(0)
-        w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = max(1, min(K, 4000) // n_sets)
-        with torch.cuda.stream(s.compute):
-            for _ in range(3):
-                gw.replay()
-            w0.record(s.compute)
-            for _ in range(reps):
-                gw.replay()
-            w1.record(s.compute)
-        torch.cuda.synchronize()
-        warm_us = w0.elapsed_time(w1) * 1e3 / (reps * n_sets * len(sets[0]))
+        warm_ms, n_warm = time_graph(gw, 1)
+        warm_us = warm_ms * 1e3 / (n_warm * n_sets * calls_per_step)
+    # a bounded device-side wait that expired anywhere above invalidates the numbers
+    try:
+        status_words = lb.pool_check_status(s.pool, s.compute)
+    except lb.LoraError:
+        status_words = [int(v) for v in s.status()]
     clocks = sampler.stop() if rank == 0 else None
 
     # swap-in on the side stream while steps run (config 4: 16 misses per step)
@@ -469,17 +485,21 @@ def main():
         lb.apply_host(s.pool, tp0, 1 if sgmv else 0, xh[c], ybh[c], yh[c], sh, T, wl.tile_m, wl.long_min,
                       L["x"], L["yb"], L["y"], L["sidx"], L["meta"], L["ws"], L["stream"])
 
-    for i in range(4):
-        e2e_step(i)
-    torch.cuda.synchronize()
+    def e2e_run(n):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for i in range(n):
+            e2e_step(i)
+        for L in lanes:
+            L["stream"].synchronize()
+        return time.perf_counter() - t0
+
+    e2e_run(8)
+    # as many steps as make the region last 0.2 s, at least the number asked for
+    Ke = all_ranks_max_int(max(Ke, int(np.ceil(0.2 / max(e2e_run(8) / 8, 1e-6)))))
     if world > 1:
         dist.barrier()
-    t0 = time.perf_counter()
-    for i in range(Ke):
-        e2e_step(i)
-    for L in lanes:
-        L["stream"].synchronize()
-    e2e_s = max_over_ranks(time.perf_counter() - t0, dev)
+    e2e_s = max_over_ranks(e2e_run(Ke), dev)
     h2d = 2 * T * (d_in0 + d_out0) + 4 * T
     d2h = 2 * T * d_out0
 
@@ -496,18 +516,20 @@ def main():
     fused = tuning.get(0) != 1
     line = {
         "metric": METRIC, "value": whole_job_value(world, T, K, ms), "unit": UNIT, "n_gpus": world,
-        "steps": K, "warmup": args.warmup, "ms_per_step": ms / K, "higher_is_better": True,
+        "steps": K_req, "steps_timed": K, "warmup": args.warmup, "ms_per_step": ms / K,
+        "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "accumulate": "fp32",
         "data": "synthetic",
         "config": {
-            "workload": WORKLOAD_TEXT[cfg] + " (%d tokens, %d distinct adapters)" % (T, len(wl.distinct_slots())),
+            "workload": workload_text(cfg, wl),
             "step": "lora_build_segments + %d x %s, one %s" % (
                 calls_per_step, "lora_sgmv_apply" if sgmv else "lora_bgmv_apply (grouped)",
                 "layer step" if cfg != 4 else "32-layer step (tokens/s per layer step = value x 32)"),
             "cache": ("cold: %d rotating input/weight sets (%.0f MB touched per rotation, L2 is 126 MB)"
                       % (n_sets, n_sets * alg / 1e6)) if n_sets > 1 else
                      "cold: one step touches %.0f MB, more than the 126 MB L2" % (alg / 1e6),
-            "launch": "CUDA graph of %d consecutive step(s) replayed" % n_sets,
+            "launch": "CUDA graph of %d consecutive step(s); every timed region is whole replays of a "
+                      "graph already replayed three times, repeated for at least %.0f ms" % (n_sets, MIN_REGION_MS),
             "multi_gpu": "independent replicas, no collective",
         },
         "roofline": {
@@ -527,9 +549,12 @@ def main():
                 "d2h_bytes_per_step": d2h, "api": "lora_apply_host (first projection of the step), two streams used alternately",
                 "steps": Ke},
         "gpu_launches": int(launches),
+        "device_status_words": status_words,
         "clocks": clocks,
         "paper_context": PAPER_CONTEXT,
     }
+    if status_words[1] != 0:
+        line["invalid"] = "a bounded device-side wait expired during the run (status word 1 = %d)" % status_words[1]
     if swap is not None:
         line["swap_in"] = swap
     if not args.no_cpu_baseline:

@@ -47,12 +47,12 @@ typedef enum {
     LORA_ERR_SHAPE = 2,            /* dimension not a multiple of 8, negative sizes */
     LORA_ERR_SLOT_RANGE = 3,       /* slot >= num_slots or < 0 */
     LORA_ERR_RANK = 4,             /* rank < 1 or rank > r_max */
-    LORA_ERR_NOT_LOADED = 5,       /* operation needs an occupied slot */
-    LORA_ERR_BUSY = 6,             /* reserved for hazards the host can see */
+    LORA_ERR_NOT_LOADED = 5,       /* operation needs an occupied slot (slot policy calls) */
+    LORA_ERR_BUSY = 6,             /* every candidate slot is pinned by an in-flight batch */
     LORA_ERR_BUFFER_TOO_SMALL = 7, /* caller buffer smaller than the matching *_bytes query */
     LORA_ERR_NOT_PINNED = 8,       /* host adapter memory is pageable */
     LORA_ERR_CUDA = 9,             /* a CUDA runtime call failed: see lora_last_cuda_error() */
-    LORA_ERR_TIMEOUT = 10          /* a bounded device-side wait expired (device status word) */
+    LORA_ERR_TIMEOUT = 10          /* a bounded device-side wait expired (lora_pool_check_status) */
 } lora_status_t;
 
 const char *lora_status_string(lora_status_t s);
@@ -148,6 +148,22 @@ lora_status_t lora_pool_slot_info(const lora_pool_t *pool, int32_t slot, int32_t
 lora_status_t lora_pool_poll_status(lora_pool_t *pool, int32_t *host_out, void *stream);
 lora_status_t lora_pool_reset_status(lora_pool_t *pool, void *stream);
 
+/* The one call that waits: copies the status words back on `stream`, synchronises that stream and
+ * returns LORA_ERR_TIMEOUT when word 1 is non-zero (some block of some kernel gave up a bounded
+ * wait and stored no result for its rows: the outputs of the applies queued since the last reset
+ * are not to be trusted), LORA_OK otherwise.  words_out (host, [4]) may be NULL.  The apply calls
+ * themselves are asynchronous and cannot report this; call it wherever a step's results are
+ * consumed on the host, or once per step in a server loop. */
+lora_status_t lora_pool_check_status(lora_pool_t *pool, void *stream, int32_t *words_out);
+
+/* Exercises the time-out path without disturbing anything: launches ONE block that polls an
+ * mbarrier nobody completes, `polls` times (1 .. 2^20), then records the expiry in status word 1
+ * exactly as the apply kernels do and returns without writing *witness_dev (dev int32, may be
+ * NULL; it is written only if the wait had succeeded).  For tests and for monitoring code that
+ * wants to see its own alarm fire. */
+lora_status_t lora_pool_selftest_wait_expiry(lora_pool_t *pool, int32_t polls, int32_t *witness_dev,
+                                             void *stream);
+
 /* Tuning knobs, for measurement (0 = the default behaviour for every key):
  *   key 0  apply path: 1 = two-phase CUDA-core kernels with the fp32 workspace
  *   key 1  fused kernel: blocks per cluster (1, 2, 4, 8)
@@ -159,6 +175,63 @@ lora_status_t lora_pool_reset_status(lora_pool_t *pool, void *stream);
  *   key 7  segment builder: 1 = one warp per slot also for long batches
  * Keys outside 0 .. 7 -> INVALID_ARG. */
 lora_status_t lora_pool_set_tuning(lora_pool_t *pool, int32_t key, int32_t value);
+
+/* ----------------------------------------------------------------------------------------
+ * Slot policy and pool sizing (paper Section 1: adapters move between CPU and GPU memory
+ * according to their usage; Section 2.2: A_max slots of one footprint S_max; Section 5: the
+ * adapter-cache stage of a step loads what the scheduled batch needs).  Host-side bookkeeping
+ * only: no CUDA call is made, and a policy object is independent of any pool.  Adapter ids are
+ * the caller's non-negative 64-bit keys.  "Least recently used" follows a logical clock advanced
+ * by every use, so decisions are a deterministic function of the call sequence.  A pinned slot
+ * (pin count > 0: an in-flight batch's metadata references it) is never chosen as a victim.
+ * Not thread-safe.
+ * -------------------------------------------------------------------------------------- */
+typedef struct lora_policy lora_policy_t;
+lora_status_t lora_policy_create(int32_t num_slots, lora_policy_t **out);
+lora_status_t lora_policy_destroy(lora_policy_t *policy);
+/* *slot_out = the slot holding the adapter, or -1. */
+lora_status_t lora_policy_lookup(const lora_policy_t *policy, int64_t adapter, int32_t *slot_out);
+/* What a slot holds (-1: empty) and its pin count; either pointer may be NULL. */
+lora_status_t lora_policy_slot(const lora_policy_t *policy, int32_t slot, int64_t *adapter_out,
+                               int32_t *pins_out);
+/* Marks the slot most recently used.  Errors: SLOT_RANGE, NOT_LOADED (empty slot). */
+lora_status_t lora_policy_touch(lora_policy_t *policy, int32_t slot);
+/* Pin / unpin the n slots of a host array (a slot named twice is pinned twice).  All or nothing.
+ * Errors: SLOT_RANGE, NOT_LOADED (pin of an empty slot), INVALID_ARG (unpin below zero). */
+lora_status_t lora_policy_pin(lora_policy_t *policy, const int32_t *slots_host, int32_t n);
+lora_status_t lora_policy_unpin(lora_policy_t *policy, const int32_t *slots_host, int32_t n);
+/* The slot to fill next: the lowest empty unpinned slot, else the unpinned slot used longest ago
+ * (ties: lowest index); *evicted_out (may be NULL) = the adapter it holds now, or -1.  Changes
+ * nothing.  Errors: BUSY (every slot is pinned). */
+lora_status_t lora_policy_choose_victim(const lora_policy_t *policy, int32_t *slot_out,
+                                        int64_t *evicted_out);
+/* Records that `adapter` now lives in `slot` (after lora_pool_load_slot), replacing what was
+ * there, and marks it used.  Errors: SLOT_RANGE, BUSY (slot pinned), INVALID_ARG (the adapter is
+ * resident in another slot). */
+lora_status_t lora_policy_assign(lora_policy_t *policy, int32_t slot, int64_t adapter);
+/* Records that the slot is empty (after lora_pool_evict_slot).  Errors: NOT_LOADED, BUSY. */
+lora_status_t lora_policy_release(lora_policy_t *policy, int32_t slot);
+/* The adapter-cache stage for one batch: adapters[i] is request i's adapter (-1: none).
+ * Writes slot_idx_out[i] (host, [n]; -1 for requests without adapter) and the loads the caller
+ * has to queue with lora_pool_load_slot before the batch's metadata is built: miss_slots_out[k],
+ * miss_adapters_out[k], k < *n_miss_out, in order of first appearance in the batch.  Victims are
+ * chosen as by lora_policy_choose_victim among slots the batch itself does not use; every slot of
+ * the batch is marked used.  On error nothing has changed.
+ * Errors: BUSY (more distinct adapters than slots that are free or may be evicted: the scheduler
+ * has to defer requests, the A_max limit of paper Section 5), BUFFER_TOO_SMALL (miss_cap). */
+lora_status_t lora_policy_admit(lora_policy_t *policy, const int64_t *adapters, int32_t n,
+                                int32_t *slot_idx_out, int32_t *miss_slots_out,
+                                int64_t *miss_adapters_out, int32_t miss_cap, int32_t *n_miss_out);
+/* Counters since creation: distinct resident adapters found per batch, loads asked for, adapters
+ * displaced.  Any pointer may be NULL. */
+lora_status_t lora_policy_stats(const lora_policy_t *policy, int64_t *hits, int64_t *misses,
+                                int64_t *evictions);
+
+/* Sizing: the largest num_slots (A_max) whose pool fits in bytes_budget for these targets at this
+ * r_max (S_max), and the bytes one more slot costs.  Errors: BUFFER_TOO_SMALL (not even one slot),
+ * plus those of lora_pool_bytes. */
+lora_status_t lora_pool_plan(size_t bytes_budget, const lora_target_t *targets, int32_t num_targets,
+                             int32_t r_max, int32_t *num_slots_out, size_t *bytes_per_slot_out);
 
 /* ----------------------------------------------------------------------------------------
  * Segment metadata (several adapters are served inside one batch, paper Section 2.2; each

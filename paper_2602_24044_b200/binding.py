@@ -28,6 +28,10 @@ EXPORTS = [
     "lora_pool_poll_status", "lora_pool_reset_status", "lora_pool_set_tuning",
     "lora_segments_bytes", "lora_build_segments", "lora_workspace_bytes",
     "lora_bgmv_apply", "lora_sgmv_apply", "lora_apply_host", "lora_bgmv_apply_static",
+    "lora_pool_check_status", "lora_pool_selftest_wait_expiry", "lora_pool_plan",
+    "lora_policy_create", "lora_policy_destroy", "lora_policy_lookup", "lora_policy_slot",
+    "lora_policy_touch", "lora_policy_pin", "lora_policy_unpin", "lora_policy_choose_victim",
+    "lora_policy_assign", "lora_policy_release", "lora_policy_admit", "lora_policy_stats",
 ]
 STATIC_SCRATCH_BYTES = 2 * 1024 * 1024
 
@@ -106,6 +110,23 @@ def _lib():
             "lora_bgmv_apply_static": [vp, i32, vp, i64, vp, i64, vp, i64, vp, i32, vp, vp],
             "lora_apply_host": [vp, i32, i32, vp, vp, vp, vp, i32, i32, i32,
                                 ctypes.POINTER(_StepBuffers), vp],
+            "lora_pool_check_status": [vp, vp, ctypes.POINTER(i32)],
+            "lora_pool_selftest_wait_expiry": [vp, i32, vp, vp],
+            "lora_pool_plan": [sz, ctypes.POINTER(_Target), i32, i32, ctypes.POINTER(i32),
+                               ctypes.POINTER(sz)],
+            "lora_policy_create": [i32, ctypes.POINTER(vp)],
+            "lora_policy_destroy": [vp],
+            "lora_policy_lookup": [vp, i64, ctypes.POINTER(i32)],
+            "lora_policy_slot": [vp, i32, ctypes.POINTER(i64), ctypes.POINTER(i32)],
+            "lora_policy_touch": [vp, i32],
+            "lora_policy_pin": [vp, ctypes.POINTER(i32), i32],
+            "lora_policy_unpin": [vp, ctypes.POINTER(i32), i32],
+            "lora_policy_choose_victim": [vp, ctypes.POINTER(i32), ctypes.POINTER(i64)],
+            "lora_policy_assign": [vp, i32, i64],
+            "lora_policy_release": [vp, i32],
+            "lora_policy_admit": [vp, ctypes.POINTER(i64), i32, ctypes.POINTER(i32),
+                                  ctypes.POINTER(i32), ctypes.POINTER(i64), i32, ctypes.POINTER(i32)],
+            "lora_policy_stats": [vp, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(i64)],
         }
         for name, args in sigs.items():
             fn = getattr(lib, name)
@@ -228,6 +249,106 @@ def pool_poll_status(pool: int, host_out, stream=None) -> None:
 
 def pool_reset_status(pool: int, stream=None) -> None:
     _check(_lib().lora_pool_reset_status(pool, _stream(stream)), "lora_pool_reset_status")
+
+
+def pool_check_status(pool: int, stream=None):
+    """Synchronises `stream`; returns the four status words.  Raises LoraError(10) when a bounded
+    device-side wait has expired since the last reset."""
+    w = (ctypes.c_int32 * 4)()
+    _check(_lib().lora_pool_check_status(pool, _stream(stream), w), "lora_pool_check_status")
+    return [int(v) for v in w]
+
+
+def pool_selftest_wait_expiry(pool: int, polls: int, witness_dev=None, stream=None) -> None:
+    _check(_lib().lora_pool_selftest_wait_expiry(pool, int(polls), _ptr(witness_dev),
+                                                 _stream(stream)), "lora_pool_selftest_wait_expiry")
+
+
+def pool_plan(bytes_budget: int, targets: Sequence, r_max: int):
+    """(num_slots that fit in bytes_budget, bytes one slot costs)."""
+    arr = (_Target * len(targets))(*[_Target(int(a), int(b)) for a, b in targets])
+    n, per = ctypes.c_int32(0), ctypes.c_size_t(0)
+    _check(_lib().lora_pool_plan(int(bytes_budget), arr, len(targets), int(r_max), ctypes.byref(n),
+                                 ctypes.byref(per)), "lora_pool_plan")
+    return int(n.value), int(per.value)
+
+
+# slot policy (host-side bookkeeping, no CUDA call)
+def policy_create(num_slots: int) -> int:
+    out = ctypes.c_void_p(None)
+    _check(_lib().lora_policy_create(int(num_slots), ctypes.byref(out)), "lora_policy_create")
+    return int(out.value)
+
+
+def policy_destroy(policy: int) -> None:
+    _check(_lib().lora_policy_destroy(policy), "lora_policy_destroy")
+
+
+def policy_lookup(policy: int, adapter: int) -> int:
+    out = ctypes.c_int32(0)
+    _check(_lib().lora_policy_lookup(policy, int(adapter), ctypes.byref(out)), "lora_policy_lookup")
+    return int(out.value)
+
+
+def policy_slot(policy: int, slot: int):
+    a, p = ctypes.c_int64(0), ctypes.c_int32(0)
+    _check(_lib().lora_policy_slot(policy, int(slot), ctypes.byref(a), ctypes.byref(p)),
+           "lora_policy_slot")
+    return int(a.value), int(p.value)
+
+
+def policy_touch(policy: int, slot: int) -> None:
+    _check(_lib().lora_policy_touch(policy, int(slot)), "lora_policy_touch")
+
+
+def _i32_array(values):
+    return (ctypes.c_int32 * max(len(values), 1))(*[int(v) for v in values])
+
+
+def policy_pin(policy: int, slots: Sequence[int]) -> None:
+    _check(_lib().lora_policy_pin(policy, _i32_array(slots), len(slots)), "lora_policy_pin")
+
+
+def policy_unpin(policy: int, slots: Sequence[int]) -> None:
+    _check(_lib().lora_policy_unpin(policy, _i32_array(slots), len(slots)), "lora_policy_unpin")
+
+
+def policy_choose_victim(policy: int):
+    """(slot, adapter it holds now or -1)."""
+    s, a = ctypes.c_int32(0), ctypes.c_int64(0)
+    _check(_lib().lora_policy_choose_victim(policy, ctypes.byref(s), ctypes.byref(a)),
+           "lora_policy_choose_victim")
+    return int(s.value), int(a.value)
+
+
+def policy_assign(policy: int, slot: int, adapter: int) -> None:
+    _check(_lib().lora_policy_assign(policy, int(slot), int(adapter)), "lora_policy_assign")
+
+
+def policy_release(policy: int, slot: int) -> None:
+    _check(_lib().lora_policy_release(policy, int(slot)), "lora_policy_release")
+
+
+def policy_admit(policy: int, adapters: Sequence[int], miss_cap: Optional[int] = None):
+    """(slot_idx int32 array, [(slot, adapter) to load, ...]) for one batch of requests."""
+    n = len(adapters)
+    cap = n if miss_cap is None else int(miss_cap)
+    ids = (ctypes.c_int64 * max(n, 1))(*[int(a) for a in adapters])
+    sidx = (ctypes.c_int32 * max(n, 1))()
+    ms = (ctypes.c_int32 * max(cap, 1))()
+    ma = (ctypes.c_int64 * max(cap, 1))()
+    nm = ctypes.c_int32(0)
+    _check(_lib().lora_policy_admit(policy, ids, n, sidx, ms, ma, cap, ctypes.byref(nm)),
+           "lora_policy_admit")
+    return (np.array(sidx[:n], dtype=np.int32),
+            [(int(ms[k]), int(ma[k])) for k in range(nm.value)])
+
+
+def policy_stats(policy: int):
+    h, m, e = ctypes.c_int64(0), ctypes.c_int64(0), ctypes.c_int64(0)
+    _check(_lib().lora_policy_stats(policy, ctypes.byref(h), ctypes.byref(m), ctypes.byref(e)),
+           "lora_policy_stats")
+    return int(h.value), int(m.value), int(e.value)
 
 
 def pool_set_tuning(pool: int, key: int, value: int) -> None:

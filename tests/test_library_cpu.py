@@ -41,7 +41,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_status_strings():
     assert lb.status_string(0) == "ok"
-    seen = {lb.status_string(i) for i in range(11)}
+    seen = {lb.status_string(i) for i in range(11)}   # every code has its own text
     assert len(seen) == 11 and "unknown status" not in seen
     assert lb.status_string(99) == "unknown status"
 
