@@ -83,8 +83,9 @@ typedef struct {
     size_t device_buf_bytes;
 } lora_pool_desc_t;
 
-/* Bytes of device memory a pool of this shape needs (control block + transpose staging +
- * num_slots slots of r_max rows for every target's A and B).  device_buf is ignored. */
+/* Bytes of device memory a pool of this shape needs (control block with the slot table and the
+ * targets' tensor maps + transpose staging + num_slots slots of r_max rows for every target's
+ * A and B).  device_buf is ignored. */
 lora_status_t lora_pool_bytes(const lora_pool_desc_t *desc, size_t *bytes);
 
 /* Creates the host handle and clears the pool's control block (slot table: all slots empty;
@@ -173,7 +174,9 @@ lora_status_t lora_pool_selftest_wait_expiry(lora_pool_t *pool, int32_t polls, i
  *   key 5  fused kernel: stages of the shared-memory ring (2 .. 4)
  *   key 6  fused kernel: 1 = partial sums always fetched from the cluster's blocks, never pushed
  *   key 7  segment builder: 1 = one warp per slot also for long batches
- * Keys outside 0 .. 7 -> INVALID_ARG. */
+ *   key 8  fused kernel: 1 = no L2 hints ahead of the shared-memory ring
+ *   key 9  fused kernel: share (1 .. 99 %) of the resident clusters one launch may take
+ * Keys outside 0 .. 15 -> INVALID_ARG. */
 lora_status_t lora_pool_set_tuning(lora_pool_t *pool, int32_t key, int32_t value);
 
 /* ----------------------------------------------------------------------------------------
@@ -290,6 +293,29 @@ lora_status_t lora_bgmv_apply(lora_pool_t *pool, int32_t target,
                               const int32_t *slot_idx_dev, int32_t T,
                               const void *meta_dev_or_null,
                               void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Several projections of ONE decode batch in one launch (paper Section 2.2: the adapters of a
+ * batch are served together through kernel-level work; Section 8.1: the models carry LoRA on all
+ * their attention and MLP projections): q/k/v, or gate/up, or all seven adapted projections of a
+ * layer when the caller has their inputs ready.  Every item is what one lora_bgmv_apply call would
+ * take; all items share the batch (slot_idx_dev, T) and its grouped metadata, which is required.
+ * The items must be independent: no item's y may overlap another item's x, y_base or y (an item's
+ * own y may equal its y_base); items may share x.  The launch walks the units of item 0 first,
+ * then item 1, ...: list wide projections first for the best balance.  Results are bit-identical
+ * to n_items separate lora_bgmv_apply calls.
+ * n_items in 1 .. LORA_MULTI_MAX.  Errors: those of lora_bgmv_apply, per item.
+ */
+#define LORA_MULTI_MAX 8
+typedef struct {
+    int32_t target;
+    const void *x;       int64_t ldx;    /* dev bf16 [T, d_in]  */
+    const void *y_base;  int64_t ldyb;   /* dev bf16 [T, d_out] */
+    void *y;             int64_t ldy;    /* dev bf16 [T, d_out] */
+} lora_apply_item_t;
+lora_status_t lora_bgmv_apply_multi(lora_pool_t *pool, const lora_apply_item_t *items, int32_t n_items,
+                                    const int32_t *slot_idx_dev, int32_t T, const void *meta_dev,
+                                    void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * lora_bgmv_apply for callers that cannot hand over a workspace (the paper has no counterpart;

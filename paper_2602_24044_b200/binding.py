@@ -28,7 +28,7 @@ EXPORTS = [
     "lora_pool_poll_status", "lora_pool_reset_status", "lora_pool_set_tuning",
     "lora_segments_bytes", "lora_build_segments", "lora_workspace_bytes",
     "lora_bgmv_apply", "lora_sgmv_apply", "lora_apply_host", "lora_bgmv_apply_static",
-    "lora_pool_check_status", "lora_pool_selftest_wait_expiry", "lora_pool_plan",
+    "lora_bgmv_apply_multi", "lora_pool_check_status", "lora_pool_selftest_wait_expiry", "lora_pool_plan",
     "lora_policy_create", "lora_policy_destroy", "lora_policy_lookup", "lora_policy_slot",
     "lora_policy_touch", "lora_policy_pin", "lora_policy_unpin", "lora_policy_choose_victim",
     "lora_policy_assign", "lora_policy_release", "lora_policy_admit", "lora_policy_stats",
@@ -60,6 +60,12 @@ class _AdapterHost(ctypes.Structure):
     _fields_ = [("rank", ctypes.c_int32), ("scale", ctypes.c_float),
                 ("A", ctypes.POINTER(ctypes.c_void_p)), ("B", ctypes.POINTER(ctypes.c_void_p)),
                 ("a_layout", ctypes.c_int32), ("trust_pinned", ctypes.c_int32)]
+
+
+class _ApplyItem(ctypes.Structure):
+    _fields_ = [("target", ctypes.c_int32), ("x", ctypes.c_void_p), ("ldx", ctypes.c_int64),
+                ("y_base", ctypes.c_void_p), ("ldyb", ctypes.c_int64),
+                ("y", ctypes.c_void_p), ("ldy", ctypes.c_int64)]
 
 
 class _StepBuffers(ctypes.Structure):
@@ -110,6 +116,7 @@ def _lib():
             "lora_bgmv_apply_static": [vp, i32, vp, i64, vp, i64, vp, i64, vp, i32, vp, vp],
             "lora_apply_host": [vp, i32, i32, vp, vp, vp, vp, i32, i32, i32,
                                 ctypes.POINTER(_StepBuffers), vp],
+            "lora_bgmv_apply_multi": [vp, ctypes.POINTER(_ApplyItem), i32, vp, i32, vp, vp, sz, vp],
             "lora_pool_check_status": [vp, vp, ctypes.POINTER(i32)],
             "lora_pool_selftest_wait_expiry": [vp, i32, vp, vp],
             "lora_pool_plan": [sz, ctypes.POINTER(_Target), i32, i32, ctypes.POINTER(i32),
@@ -384,6 +391,28 @@ def bgmv_apply(pool: int, target: int, x, ldx: int, y_base, ldyb: int, y, ldy: i
     _check(_lib().lora_bgmv_apply(pool, int(target), _ptr(x), int(ldx), _ptr(y_base), int(ldyb),
                                   _ptr(y), int(ldy), _ptr(slot_idx_dev), int(T), _ptr(meta_dev),
                                   _ptr(workspace), nbytes, _stream(stream)), "lora_bgmv_apply")
+
+
+def make_apply_items(items: Sequence):
+    """items: (target, x, ldx, y_base, ldyb, y, ldy) tuples -> a C array for bgmv_apply_multi (build
+    it once when the same launch is issued repeatedly)."""
+    arr = (_ApplyItem * max(len(items), 1))()
+    for k, (target, x, ldx, yb, ldyb, y, ldy) in enumerate(items):
+        arr[k] = _ApplyItem(int(target), _ptr(x), int(ldx), _ptr(yb), int(ldyb), _ptr(y), int(ldy))
+    return arr, len(items)
+
+
+def bgmv_apply_multi(pool: int, items, slot_idx_dev, T: int, meta_dev, workspace,
+                     workspace_bytes_: Optional[int] = None, stream=None) -> None:
+    """Several projections of one decode batch in one launch; `items` as for make_apply_items (or
+    its result)."""
+    arr, n = items if isinstance(items, tuple) and len(items) == 2 and not isinstance(items[0], tuple) \
+        else make_apply_items(items)
+    nbytes = (_nbytes(workspace) if workspace is not None else 0) \
+        if workspace_bytes_ is None else workspace_bytes_
+    _check(_lib().lora_bgmv_apply_multi(pool, arr, n, _ptr(slot_idx_dev), int(T), _ptr(meta_dev),
+                                        _ptr(workspace), nbytes, _stream(stream)),
+           "lora_bgmv_apply_multi")
 
 
 def bgmv_apply_static(pool: int, target: int, x, ldx: int, y_base, ldyb: int, y, ldy: int,

@@ -109,6 +109,51 @@ lora_status_t lora_bgmv_apply(lora_pool_t *pool, int32_t target, const void *x, 
                         workspace, workspace_bytes, (cudaStream_t)stream, false);
 }
 
+lora_status_t lora_bgmv_apply_multi(lora_pool_t *pool, const lora_apply_item_t *items, int32_t n_items,
+                                    const int32_t *slot_idx_dev, int32_t T, const void *meta,
+                                    void *workspace, size_t workspace_bytes, void *stream) {
+    if (!pool || !items || n_items < 1 || n_items > LORA_MULTI_MAX) return LORA_ERR_INVALID_ARG;
+    if (T < 0) return LORA_ERR_SHAPE;
+    for (int32_t i = 0; i < n_items; ++i) {
+        const lora_apply_item_t &it = items[i];
+        lora_status_t s = check_apply_args(pool, it.target, it.x, it.ldx, it.y_base, it.ldyb, it.y, it.ldy, T);
+        if (s != LORA_OK) return s;
+    }
+    if (T == 0) return LORA_OK;
+    if (!meta) return LORA_ERR_INVALID_ARG;
+    int32_t tile_m = 1;
+    if (!pool->find_meta(meta, T, &tile_m)) return LORA_ERR_INVALID_ARG;
+    // independence: nothing an item writes may be read or written by another item
+    for (int32_t i = 0; i < n_items; ++i) {
+        const lora_target_t &ti = pool->targets[items[i].target];
+        const size_t ny = ((size_t)(T - 1) * items[i].ldy + ti.d_out) * 2;
+        for (int32_t j = 0; j < n_items; ++j) {
+            if (j == i) continue;
+            const lora_target_t &tj = pool->targets[items[j].target];
+            if (ranges_overlap(items[i].y, ny, items[j].x, ((size_t)(T - 1) * items[j].ldx + tj.d_in) * 2) ||
+                ranges_overlap(items[i].y, ny, items[j].y_base, ((size_t)(T - 1) * items[j].ldyb + tj.d_out) * 2) ||
+                ranges_overlap(items[i].y, ny, items[j].y, ((size_t)(T - 1) * items[j].ldy + tj.d_out) * 2))
+                return LORA_ERR_INVALID_ARG;
+        }
+    }
+    if (!workspace || workspace_bytes < (size_t)T * rank_bucket(pool->r_max) * sizeof(float))
+        return LORA_ERR_BUFFER_TOO_SMALL;
+    DeviceGuard guard(pool->device);
+    if (!guard.ok) return cuda_fail(cudaErrorInvalidDevice);
+    ApplyParams P[LORA_MULTI_MAX];
+    for (int32_t i = 0; i < n_items; ++i)
+        fill_apply_params(pool, P[i], items[i].target, items[i].x, items[i].ldx, items[i].y_base,
+                          items[i].ldyb, items[i].y, items[i].ldy, slot_idx_dev, T, meta, tile_m);
+    if (pool->tuning[0] == 1) {   // the two-phase baseline has no multi-projection form
+        for (int32_t i = 0; i < n_items; ++i) {
+            lora_status_t s = launch_twophase(pool, P[i], workspace, workspace_bytes, (cudaStream_t)stream);
+            if (s != LORA_OK) return s;
+        }
+        return LORA_OK;
+    }
+    return launch_fused_items(pool, P, n_items, (cudaStream_t)stream);
+}
+
 lora_status_t lora_sgmv_apply(lora_pool_t *pool, int32_t target, const void *x, int64_t ldx,
                               const void *y_base, int64_t ldyb, void *y, int64_t ldy,
                               const void *meta, int32_t T, void *workspace, size_t workspace_bytes,

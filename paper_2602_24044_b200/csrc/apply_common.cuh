@@ -137,6 +137,9 @@ static inline int32_t next_pow2(int32_t v) {
 lora_status_t launch_twophase(lora_pool_t *pool, ApplyParams &P, void *workspace,
                               size_t workspace_bytes, cudaStream_t stream);
 lora_status_t launch_fused(lora_pool_t *pool, ApplyParams &P, cudaStream_t stream);
+lora_status_t launch_fused_items(lora_pool_t *pool, const ApplyParams *items, int32_t n_items,
+                                 cudaStream_t stream);
+lora_status_t build_fused_maps(lora_pool_t *pool);
 lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, void *workspace,
                                    size_t workspace_bytes, cudaStream_t stream, bool *handled);
 lora_status_t launch_build_segments(lora_pool_t *pool, const int32_t *slot_idx_dev, int32_t T,

@@ -137,14 +137,17 @@ struct lora_pool {
     cudaEvent_t fence = nullptr;        // compute -> load ordering
     int32_t sm_count = 148;
     uint32_t bucket_mask = 0;           // rank buckets (8/16/32/64 -> bits 0..3) ever loaded into a slot
-    int32_t tuning[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    // Tensor maps of the fused kernel, built on first use: per target, 8 for A and 8 for B (one
-    // per number of rank rows 8, 16, .. 64 a tile load fetches).
-    struct alignas(64) TargetMaps {
-        CUtensorMap a[8], b[8];
+    int32_t tuning[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+    // Tensor maps of the fused kernel in the pool's device buffer, written at creation: per
+    // target 8 for A and 8 for B (one per number of rank rows 8, 16, .. 64 a tile load fetches).
+    CUtensorMap *maps_dev = nullptr;
+    // What the fused kernel's launcher has set or asked for this pool's device (dynamic
+    // shared-memory limit, resident clusters), per kernel variant; part of the handle, so pools
+    // used from different threads share nothing.
+    struct FusedLaunchCache {
+        int32_t attr_smem = 0, occ_smem = 0, occ_c = 0, occ_clusters = 0;
     };
-    std::vector<TargetMaps> fused_maps;
-    std::vector<uint8_t> fused_maps_ready;
+    FusedLaunchCache fused_cache[2];
 
     // Shapes of the metadata tables built through this handle (the table itself lives on the
     // device; apply calls need T and tile_m on the host to size their grids).

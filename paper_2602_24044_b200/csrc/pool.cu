@@ -3,7 +3,7 @@
 // Section 5 whose cost Eq. 1 calls Lat_load).
 #include <new>
 
-#include "common.cuh"
+#include "apply_common.cuh"
 
 namespace lora {
 
@@ -13,7 +13,7 @@ std::atomic<int64_t> g_launch_count{0};
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct PoolLayout {
-    size_t off_status, off_table, off_staging, off_weights, bytes;
+    size_t off_status, off_table, off_maps, off_staging, off_weights, bytes;
     size_t staging_elems;
     int64_t slot_stride;   // elements
 };
@@ -41,7 +41,8 @@ static PoolLayout pool_layout(const lora_pool_desc_t *d) {
     L.staging_elems = (size_t)max_d_in * d->r_max;
     L.off_status = 0;
     L.off_table = 256;
-    L.off_staging = align_up(L.off_table + sizeof(SlotEntry) * (size_t)d->num_slots, 256);
+    L.off_maps = align_up(L.off_table + sizeof(SlotEntry) * (size_t)d->num_slots, 256);
+    L.off_staging = align_up(L.off_maps + (size_t)d->num_targets * 16 * sizeof(CUtensorMap), 256);
     L.off_weights = align_up(L.off_staging + L.staging_elems * 2, 256);
     // 256 bytes of slack after the last slot: tiled loads of 64-column blocks may start inside
     // the last row of the last matrix and run up to 126 bytes past its end
@@ -133,6 +134,7 @@ lora_status_t lora_pool_create(const lora_pool_desc_t *desc, lora_pool_t **out) 
     p->bytes = L.bytes;
     p->status_dev = (int32_t *)(p->base + L.off_status);
     p->table_dev = (SlotEntry *)(p->base + L.off_table);
+    p->maps_dev = (CUtensorMap *)(p->base + L.off_maps);
     p->staging_dev = (__nv_bfloat16 *)(p->base + L.off_staging);
     p->staging_elems = L.staging_elems;
     p->weights_dev = (__nv_bfloat16 *)(p->base + L.off_weights);
@@ -152,13 +154,18 @@ lora_status_t lora_pool_create(const lora_pool_desc_t *desc, lora_pool_t **out) 
     p->table_host.assign(p->num_slots, empty);
     p->ready.assign(p->num_slots, nullptr);
     cudaError_t e = cudaEventCreateWithFlags(&p->fence, cudaEventDisableTiming);
-    if (e == cudaSuccess) e = cudaMemset(p->base, 0, L.off_staging);   // status + table
+    if (e == cudaSuccess) e = cudaMemset(p->base, 0, L.off_staging);   // status, table, tensor maps
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount,
                                                      desc->device);
     if (e != cudaSuccess) {
         if (p->fence) cudaEventDestroy(p->fence);
         delete p;
         return cuda_fail(e);
+    }
+    if ((s = build_fused_maps(p)) != LORA_OK) {
+        cudaEventDestroy(p->fence);
+        delete p;
+        return s;
     }
     *out = p;
     return LORA_OK;
@@ -348,7 +355,7 @@ lora_status_t lora_pool_reset_status(lora_pool_t *pool, void *stream) {
 }
 
 lora_status_t lora_pool_set_tuning(lora_pool_t *pool, int32_t key, int32_t value) {
-    if (!pool || key < 0 || key >= 8) return LORA_ERR_INVALID_ARG;
+    if (!pool || key < 0 || key >= 16) return LORA_ERR_INVALID_ARG;
     pool->tuning[key] = value;
     return LORA_OK;
 }
