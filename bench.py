@@ -57,6 +57,12 @@ def parse_args():
                     help="apply path: 0 fused cluster kernel (default), 1 two-phase kernels")
     ap.add_argument("--cluster", type=int, default=None, help="fused path: cluster size 1/2/4/8")
     ap.add_argument("--tile-m", type=int, default=None, help="rows per tile of the segment metadata")
+    ap.add_argument("--multi", default="layer", choices=["off", "groups", "layer"],
+                    help="config 4: projections per launch: off = one lora_bgmv_apply each; groups = "
+                         "{q,k,v} {o} {gate,up} {down} (the projections whose inputs exist together in a "
+                         "transformer layer); layer = all seven of a layer in one lora_bgmv_apply_multi")
+    ap.add_argument("--layers", type=int, default=32,
+                    help="config 4: transformer layers in the step (fewer only for profiling captures)")
     ap.add_argument("--tune", nargs="*", default=[], metavar="KEY=VALUE",
                     help="lora_pool_set_tuning pairs, e.g. 2=1 (no programmatic dependent launch)")
     return ap.parse_args()
@@ -233,11 +239,11 @@ def workload_text(cfg, wl):
     return WORKLOAD_TEXT[cfg] + " (%d tokens, %d distinct adapters)" % (wl.T, len(wl.distinct_slots()))
 
 
-def case_workload(cfg):
+def case_workload(cfg, layers=32):
     """The workload object of a configuration, with the rotation of independent copies that keeps
     every step cold in L2 for the small ones."""
     from paper_2602_24044_b200 import workloads as W
-    wl = W.make_config(cfg)
+    wl = W.make_config(cfg, layers=layers) if cfg == 4 else W.make_config(cfg)
     rotation = 1
     if cfg in (0, 1):
         rotation = ROTATION
@@ -276,7 +282,7 @@ def main():
         dist.barrier()
 
     cfg = args.config
-    wl, rotation, n_proj = case_workload(cfg)
+    wl, rotation, n_proj = case_workload(cfg, args.layers)
     if args.tile_m is not None:
         wl.tile_m = args.tile_m
     T = wl.T
@@ -306,11 +312,19 @@ def main():
     meta_words = lb.segments_bytes(T, wl.num_slots, wl.tile_m) // 4
     n_sets = rotation if cfg != 4 else 1
     acts = {}
+    multi = args.multi if (cfg == 4 and tuning.get(0) != 1) else "off"
+    share = {1: 0, 2: 0, 5: 4} if multi != "off" else {}     # k, v read q's input; up reads gate's
     for r in range(n_sets):
         calls = []
         for j in range(len(wl.calls) // n_sets):
             call = r * (len(wl.calls) // n_sets) + j
             key = call if cfg != 4 else call % (7 * act_sets)
+            if cfg == 4 and (call % 7) in share and key not in acts:
+                # same device tensor for the shared input, own y_base and y
+                kx = key - (call % 7) + share[call % 7]
+                _, yb_h = wl.activations(key)
+                acts[key] = (acts[kx][0], bf16_tensor(yb_h, dev),
+                             torch.empty(yb_h.shape, dtype=torch.bfloat16, device=dev))
             if key not in acts:
                 x_h, yb_h = wl.activations(key)
                 acts[key] = (bf16_tensor(x_h, dev), bf16_tensor(yb_h, dev),
@@ -322,7 +336,24 @@ def main():
     torch.cuda.synchronize()
     sgmv = wl.kind == "sgmv"
 
+    # config 4 with several projections per launch: item lists built once
+    launches_multi = None
+    if multi != "off":
+        shapes = {"layer": [[4, 5, 6, 0, 3, 1, 2]], "groups": [[0, 1, 2], [3], [4, 5], [6]]}[multi]
+        launches_multi = []
+        for layer in range(len(sets[0]) // 7):
+            for grp in shapes:
+                items = []
+                for p in grp:
+                    tp, x, yb, y = sets[0][7 * layer + p]
+                    items.append((tp, x, x.shape[1], yb, yb.shape[1], y, y.shape[1]))
+                launches_multi.append(lb.make_apply_items(items))
+
     def apply_calls(r):
+        if launches_multi is not None:
+            for items in launches_multi:
+                lb.bgmv_apply_multi(s.pool, items, s.slot_idx_dev, T, metas[r], s.ws, stream=s.compute)
+            return
         for tp, x, yb, y in sets[r]:
             if sgmv:
                 lb.sgmv_apply(s.pool, tp, x, x.shape[1], yb, yb.shape[1], y, y.shape[1], metas[r], T, s.ws,
@@ -411,8 +442,9 @@ def main():
 
     # the applies alone (dominant kernel), same rotation, for the roofline figure
     calls_per_step = len(sets[0])
+    launches_per_step = len(launches_multi) if launches_multi is not None else calls_per_step
     apply_total_ms, n_apply_rep = time_graph(g_apply, 1)
-    apply_ms = apply_total_ms / (n_apply_rep * n_sets) / calls_per_step
+    apply_ms = apply_total_ms / (n_apply_rep * n_sets) / launches_per_step
     # the same applies with ONE input / weight set replayed (small configurations: everything stays
     # in L2), reported beside the cold figure and labelled as warm
     warm_us = None
@@ -422,7 +454,7 @@ def main():
             for _ in range(n_sets):
                 apply_calls(0)
         warm_ms, n_warm = time_graph(gw, 1)
-        warm_us = warm_ms * 1e3 / (n_warm * n_sets * calls_per_step)
+        warm_us = warm_ms * 1e3 / (n_warm * n_sets * launches_per_step)
     # a bounded device-side wait that expired anywhere above invalidates the numbers
     try:
         status_words = lb.pool_check_status(s.pool, s.compute)
@@ -511,8 +543,10 @@ def main():
 
     peak, peak_kind = measured_peak()
     alg_calls = [algorithmic_bytes(wl, wl.calls[j]) for j in range(calls_per_step)]
-    alg = sum(alg_calls)
-    achieved = alg / calls_per_step / (apply_ms * 1e-3) / 1e9
+    # an input shared by several projections of a launch is counted once
+    alg = sum(alg_calls) - sum(2 * T * wl.targets[wl.calls[j]][0]
+                               for j in range(calls_per_step) if (j % 7) in share)
+    achieved = alg / launches_per_step / (apply_ms * 1e-3) / 1e9
     fused = tuning.get(0) != 1
     line = {
         "metric": METRIC, "value": whole_job_value(world, T, K, ms), "unit": UNIT, "n_gpus": world,
@@ -522,8 +556,12 @@ def main():
         "data": "synthetic",
         "config": {
             "workload": workload_text(cfg, wl),
-            "step": "lora_build_segments + %d x %s, one %s" % (
-                calls_per_step, "lora_sgmv_apply" if sgmv else "lora_bgmv_apply (grouped)",
+            "step": "lora_build_segments + %s, one %s" % (
+                "%d x lora_sgmv_apply" % calls_per_step if sgmv else
+                "%d x lora_bgmv_apply (grouped)" % calls_per_step if launches_multi is None else
+                "%d x lora_bgmv_apply_multi (%d projections; %s; q/k/v and gate/up share their input)" % (
+                    launches_per_step, calls_per_step,
+                    "one launch per layer" if multi == "layer" else "{q,k,v} {o} {gate,up} {down} per launch"),
                 "layer step" if cfg != 4 else "32-layer step (tokens/s per layer step = value x 32)"),
             "cache": ("cold: %d rotating input/weight sets (%.0f MB touched per rotation, L2 is 126 MB)"
                       % (n_sets, n_sets * alg / 1e6)) if n_sets > 1 else
@@ -539,9 +577,9 @@ def main():
             "kernel": ("shrink_kernel + expand_kernel (two launches per apply)" if not fused
                        else "tc_shrink_kernel + tc_expand_kernel + fused_kernel (one apply; tc_expand dominates)"
                        if cfg == 2 else "fused_kernel (one launch per apply, every rank)"),
-            "algorithmic_bytes_per_launch": alg / calls_per_step,
+            "algorithmic_bytes_per_launch": alg / launches_per_step,
             "us_per_launch": apply_ms * 1e3, "traffic": NCU_TRAFFIC.get(cfg) if fused else None,
-            "averaged_over": "%d applies per step" % calls_per_step,
+            "averaged_over": "%d launches per step" % launches_per_step,
             "warm_l2_us_per_launch": warm_us,
         },
         "step_GBps": alg / (ms / K * 1e-3) / 1e9,

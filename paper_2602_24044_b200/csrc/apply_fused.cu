@@ -40,6 +40,7 @@
 #include <cstring>
 
 #include "apply_common.cuh"
+#include "fused_ptx.cuh"
 
 namespace lora {
 
@@ -91,172 +92,6 @@ struct FusedParams {
 };
 
 // ---------------------------------------------------------------------------------------------
-// PTX wrappers
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) {
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void fence_mbar_init() {
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-}
-__device__ __forceinline__ void fence_proxy_async() {
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
-                 "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// barrier among the four consumer warps (the requesting warp runs on its own)
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// bounded wait: gives up after a fixed number of polls instead of spinning for ever
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
-    for (uint32_t i = 0; i < (1u << 20); ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-// global -> this block's shared memory, completion counted in bytes on the mbarrier
-__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-            smem_u32(dst)),
-        "l"(src), "r"(bytes), "r"(smem_u32(bar))
-        : "memory");
-}
-// one tile of a 4-D tensor (column in block, rank row, column block, slot) -> shared memory
-__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, int c0, int c1, int c2,
-                                            int c3, uint64_t *bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, "
-        "%3, %4, %5}], [%6];" ::"r"(smem_u32(dst)),
-        "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar))
-        : "memory");
-}
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ uint32_t cluster_nctarank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_arrive() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void cluster_wait() {
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// one arrival on the mbarrier at the same shared-memory offset in block `rank` of the cluster; the
-// arriving thread's earlier writes and reads are ordered before it (release at cluster scope)
-__device__ __forceinline__ void mbar_arrive_peer(uint64_t *local_bar, uint32_t rank) {
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local_bar)), "r"(rank));
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
-}
-// bounded wait on this block's mbarrier for arrivals from the whole cluster (acquire at cluster scope)
-__device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity) {
-    for (uint32_t i = 0; i < (1u << 20); ++i) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok)
-            : "r"(smem_u32(bar)), "r"(parity)
-            : "memory");
-        if (ok) return true;
-    }
-    return false;
-}
-// read a float at the same shared-memory offset in block `rank` of the cluster
-__device__ __forceinline__ float ld_peer_f32(uint32_t local_addr, uint32_t rank) {
-    uint32_t remote;
-    float v;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
-    return v;
-}
-// write a float at the same shared-memory offset in block `rank` of the cluster
-__device__ __forceinline__ void st_peer_f32(uint32_t local_addr, uint32_t rank, float v) {
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
-}
-// D += A(16x16, row) . B(16x8, col), bf16 inputs, fp32 accumulate
-__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
-                                         uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-        "{%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-// four 8x8 b16 matrices, transposed on the way in (rows of shared memory become MMA columns)
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-// programmatic dependent launch: let the next kernel of the stream be scheduled / wait until all
-// work queued before this kernel is complete and visible (no-ops without the launch attribute)
-__device__ __forceinline__ void griddep_launch_dependents() {
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-}
-__device__ __forceinline__ void griddep_wait() {
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-}
-__device__ __forceinline__ uint32_t lds32(const __nv_bfloat16 *p) {
-    return *reinterpret_cast<const uint32_t *>(p);
-}
-__device__ __forceinline__ uint32_t lds32b(const unsigned char *p) {
-    return *reinterpret_cast<const uint32_t *>(p);
-}
-__device__ __forceinline__ int4 ldg_int4(const int32_t *p) {
-    int4 v;
-    asm volatile("ld.global.nc.v4.s32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
-__device__ __forceinline__ int32_t ldg_int(const int32_t *p) {
-    int32_t v;
-    asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(v) : "l"(p));
-    return v;
-}
-
-// ask L2 for one tile of a 4-D tensor / for a run of bytes (hints: nothing is delivered anywhere)
-__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap *map, int c0, int c1, int c2, int c3) {
-    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(map),
-                 "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
-}
-
-// ---------------------------------------------------------------------------------------------
 // units and the record ring
 // ---------------------------------------------------------------------------------------------
 struct Unit {
@@ -270,6 +105,23 @@ struct Unit {
     bool run;            // the unit has jobs in this launch
 };
 
+// Position in the launch's unit list: unit g is unit u of projection `item`.  A cluster walks
+// g = cid, cid + G, ...; the split into (item, u) is carried along instead of divided out.
+struct Walk {
+    int32_t g, item, u;
+    __device__ __forceinline__ void start(int32_t cid, int32_t n_units) {
+        g = u = cid;
+        item = 0;
+        while (u >= n_units) { u -= n_units; ++item; }
+    }
+    __device__ __forceinline__ Walk next(int32_t G, int32_t n_units) const {
+        Walk w;
+        w.g = g + G; w.u = u + G; w.item = item;
+        while (w.u >= n_units) { w.u -= n_units; ++w.item; }
+        return w;
+    }
+};
+
 // What every part of a block needs to know about its place and progress.
 struct Ctx {
     unsigned char *smem;
@@ -278,7 +130,8 @@ struct Ctx {
     int32_t cid, G;            // cluster index, clusters in the grid
     int32_t n_units, total;    // units per projection, units of the launch
     uint32_t crank, csize;
-    int32_t cq;                // jobs consumed so far
+    int32_t st;                // ring stage of the next job (consumers: to consume, requesting warp: to fill)
+    uint32_t ph;               // how often the ring has wrapped, low bit = the stage's phase
     int32_t kp, kr;            // units whose partials this block has published / summed
     bool ok;                   // no wait has expired
 };
@@ -286,17 +139,23 @@ struct Ctx {
 __device__ __forceinline__ volatile int32_t *dead_flag(unsigned char *smem) {
     return reinterpret_cast<volatile int32_t *>(smem + SM_DEAD);
 }
+__device__ __forceinline__ void ring_advance(const FusedParams &P, Ctx &cx) {
+    if (++cx.st == P.n_stages) {
+        cx.st = 0;
+        ++cx.ph;
+    }
+}
 
 // record: {slot (-1: token without adapter, -2: past the end), position, rows | tile rows << 8 |
-// consecutive ids << 16 | rank << 17, scale bits}; g: the unit's number in the launch
-__device__ __forceinline__ Unit decode_unit(const FusedParams &P, const Ctx &cx, const int4 rec, int32_t g) {
+// consecutive ids << 16 | rank << 17, scale bits}
+__device__ __forceinline__ Unit decode_unit(const FusedParams &P, const Ctx &cx, const int4 rec, int32_t item) {
     Unit u;
     u.slot = rec.x;
     u.rows = rec.z & 0xff;
     const int32_t tile_rows = (rec.z >> 8) & 0xff, contiguous = (rec.z >> 16) & 1;
     u.rank = (rec.z >> 17) & 0x7f;
     u.scale = __int_as_float(rec.w);
-    u.item = min(g / cx.n_units, P.n_items - 1);
+    u.item = min(item, P.n_items - 1);
     const FusedItem &it = P.item[u.item];
     u.a_lo = min((int32_t)cx.crank * it.wa, it.d_in);
     u.a_hi = min(u.a_lo + it.wa, it.d_in);
@@ -319,15 +178,13 @@ struct UnitRegs {   // a record on its way from global memory to the ring (lane 
     int32_t rowid;
 };
 
-// Requests the record of the launch's unit g (g < cap bounds the addresses that may be read;
-// whether g is a real unit is decided when the record is used).
-__device__ __forceinline__ UnitRegs fetch_unit(const FusedParams &P, int32_t g, int32_t n_units, int32_t cap,
-                                               int lane) {
+// Requests the record of unit u of the batch (`valid`: the address may be read; whether the unit
+// is a real one is decided when the record is used).
+__device__ __forceinline__ UnitRegs fetch_unit(const FusedParams &P, int32_t u, bool valid, int lane) {
     UnitRegs m;
     m.rec = make_int4(-2, 0, 0, 0);
     m.rowid = 0;
-    if (g >= cap) return m;
-    const int32_t u = g % n_units;
+    if (!valid) return m;
     if (P.meta) {
         if (lane == 16) m.rec = ldg_int4(P.meta + P.moff_udesc + 4 * (int64_t)u);
         else if (lane < 16) m.rowid = ldg_int(P.meta + P.moff_uperm + 16 * (int64_t)u + lane);
@@ -348,7 +205,7 @@ __device__ __forceinline__ UnitRegs fetch_unit(const FusedParams &P, int32_t g, 
 }
 __device__ __forceinline__ void store_unit(unsigned char *smem, int32_t iter, const UnitRegs &m,
                                            bool real, int lane) {
-    unsigned char *e = smem + SM_RING + (iter % UNIT_RING) * RING_ENTRY;
+    unsigned char *e = smem + SM_RING + (iter & (UNIT_RING - 1)) * RING_ENTRY;
     if (lane == 16) *reinterpret_cast<int4 *>(e) = real ? m.rec : make_int4(-2, 0, 0, 0);
     else if (lane < 16) reinterpret_cast<int32_t *>(e + 16)[lane] = m.rowid;
 }
@@ -359,6 +216,12 @@ __device__ __forceinline__ int4 bcast_rec(const UnitRegs &m) {
     rec.z = __shfl_sync(0xffffffffu, m.rec.z, 16);
     rec.w = __shfl_sync(0xffffffffu, m.rec.w, 16);
     return rec;
+}
+// The unit count of the batch as the kernel sees it, and the launch's total.
+__device__ __forceinline__ void set_counts(const FusedParams &P, Ctx &cx, int32_t n_units) {
+    if (n_units > P.units_cap) n_units = P.units_cap;
+    cx.total = n_units * P.n_items;
+    cx.n_units = n_units < 1 ? 1 : n_units;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -420,36 +283,25 @@ __device__ __forceinline__ void producer_warp(const FusedParams &P, Ctx &cx, int
     volatile int32_t *dead = dead_flag(cx.smem);
     volatile int32_t *issued = reinterpret_cast<volatile int32_t *>(cx.smem + SM_ISSUED);
     // the unit count and (speculatively, as if the table were full) the first record, side by side
-    int32_t n_units = P.meta ? ldg_int(P.meta + H_NPIECE) : P.T;
-    UnitRegs cur = fetch_unit(P, cx.cid, P.units_cap, P.units_cap * P.n_items, lane);
-    if (n_units > P.units_cap) n_units = P.units_cap;
-    cx.total = n_units * P.n_items;
-    if (n_units < 1) n_units = 1;
-    cx.n_units = n_units;
-    if (n_units != P.units_cap && P.n_items > 1) cur = fetch_unit(P, cx.cid, n_units, cx.total, lane);
+    const int32_t n_hdr = P.meta ? ldg_int(P.meta + H_NPIECE) : P.T;
+    UnitRegs cur = fetch_unit(P, cx.cid, P.n_items == 1 && cx.cid < P.units_cap, lane);
+    set_counts(P, cx, n_hdr);
+    Walk w;
+    w.start(cx.cid, cx.n_units);
+    if (P.n_items > 1) cur = fetch_unit(P, w.u, w.g < cx.total, lane);
     int32_t q = 0, skip = 0;
     bool have_pend = false, waited = !P.early;
     Unit pend;
     int32_t pend_rowid = 0;
 
-    auto issue = [&](const Unit &un, int32_t j, int32_t rowid) {
-        const int st = q % S;
-        if (q >= S && cx.ok) {
-            cx.ok = mbar_wait(&cx.empty[st], (uint32_t)(q / S - 1) & 1u);
-            if (!cx.ok) *dead = 1;
-        }
-        if (cx.ok && !*dead) {
-            request_job(P, cx, un, j, st, rowid, lane, 0);
-            if (lane == 0) *issued = q + 1;
-        }
-        ++q;
-    };
-
     for (int32_t i = 0;; ++i) {
-        const int32_t g = cx.cid + i * cx.G;
-        if (g >= cx.total) break;
-        const UnitRegs nxt = fetch_unit(P, g + cx.G, n_units, cx.total, lane);   // the next unit's record, meanwhile
-        const Unit un = decode_unit(P, cx, bcast_rec(cur), g);
+        const bool real = w.g < cx.total;
+        if (!real && !have_pend) break;
+        const Walk wn = w.next(cx.G, cx.n_units);
+        const bool next_real = real && wn.g < cx.total;
+        const UnitRegs nxt = fetch_unit(P, wn.u, next_real, lane);   // the next unit's record, meanwhile
+        Unit un = decode_unit(P, cx, bcast_rec(cur), w.item);
+        if (!real) un.run = false;   // past the end: only the last unit's expand jobs are left
         if (i == 0) {
             if (P.early) {
                 // The kernel before this one may still be running: the pool may be read (the host
@@ -460,31 +312,46 @@ __device__ __forceinline__ void producer_warp(const FusedParams &P, Ctx &cx, int
             }
             if (P.prefetch) prefetch_unit(P, un, skip, cur.rowid, lane);
         }
-        const bool hint_next = P.prefetch && g + cx.G < cx.total;
+        const bool hint_next = P.prefetch && next_real;
         const bool hint_first = i == 0 && !waited;   // time to spare before the wait returns
-        if (hint_next && hint_first)
-            prefetch_unit(P, decode_unit(P, cx, bcast_rec(nxt), g + cx.G), 0, nxt.rowid, lane);
+        Unit un_next;
+        if (hint_next) un_next = decode_unit(P, cx, bcast_rec(nxt), wn.item);
+        if (hint_next && hint_first) prefetch_unit(P, un_next, 0, nxt.rowid, lane);
         if (!waited) {
             griddep_wait();
             waited = true;
-            for (int32_t j = 0; j < skip; ++j) request_job(P, cx, un, j, j, cur.rowid, lane, 2);
+            for (int32_t j = 0; j < skip; ++j) {
+                request_job(P, cx, un, j, j, cur.rowid, lane, 2);
+                ring_advance(P, cx);
+            }
             if (lane == 0) *issued = skip;
             q = skip;
         }
-        if (un.run)
-            for (int32_t j = (i == 0 ? skip : 0); j < un.na; ++j) issue(un, j, cur.rowid);
-        if (hint_next && !hint_first)
-            prefetch_unit(P, decode_unit(P, cx, bcast_rec(nxt), g + cx.G), 0, nxt.rowid, lane);
-        if (have_pend)
-            for (int32_t j = pend.na; j < pend.na + pend.nb; ++j) issue(pend, j, pend_rowid);
+        // this step's jobs in ring order: the unit's shrink chunks, then the pending unit's expand chunks
+        const int32_t ja = un.run ? un.na : 0, jb = have_pend ? pend.nb : 0;
+        for (int32_t k = (i == 0 ? skip : 0); k < ja + jb; ++k) {
+            if (k == ja && hint_next && !hint_first) prefetch_unit(P, un_next, 0, nxt.rowid, lane);
+            if (q >= S && cx.ok) {
+                cx.ok = mbar_wait(&cx.empty[cx.st], (cx.ph - 1u) & 1u);
+                if (!cx.ok) *dead = 1;
+            }
+            if (cx.ok && !*dead) {
+                if (k < ja) request_job(P, cx, un, k, cx.st, cur.rowid, lane, 0);
+                else request_job(P, cx, pend, pend.na + k - ja, cx.st, pend_rowid, lane, 0);
+                if (lane == 0) *issued = q + 1;
+            }
+            ++q;
+            ring_advance(P, cx);
+        }
+        if (jb == 0 && hint_next && !hint_first) prefetch_unit(P, un_next, 0, nxt.rowid, lane);
         have_pend = un.run;
         pend = un;
         pend_rowid = cur.rowid;
+        if (!real) break;
         cur = nxt;
+        w = wn;
     }
     if (!waited) griddep_wait();
-    if (have_pend)
-        for (int32_t j = pend.na; j < pend.na + pend.nb; ++j) issue(pend, j, pend_rowid);
     if (!cx.ok && lane == 0) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
 }
 
@@ -493,18 +360,17 @@ __device__ __forceinline__ void producer_warp(const FusedParams &P, Ctx &cx, int
 // ---------------------------------------------------------------------------------------------
 // wait for the data of the next job; returns its stage number
 __device__ __forceinline__ int acquire_job(const FusedParams &P, Ctx &cx) {
-    const int st = cx.cq % P.n_stages;
     if (cx.ok) {
-        cx.ok = mbar_wait(&cx.full[st], (uint32_t)(cx.cq / P.n_stages) & 1u);
+        cx.ok = mbar_wait(&cx.full[cx.st], cx.ph & 1u);
         if (!cx.ok) *dead_flag(cx.smem) = 1;
     }
-    return st;
+    return cx.st;
 }
 // this warp is done with the job's stage
 __device__ __forceinline__ void release_job(const FusedParams &P, Ctx &cx, int lane) {
     __syncwarp();
-    if (lane == 0 && cx.ok) mbar_arrive(&cx.empty[cx.cq % P.n_stages]);
-    ++cx.cq;
+    if (lane == 0 && cx.ok) mbar_arrive(&cx.empty[cx.st]);
+    ring_advance(P, cx);
 }
 
 // Shrink of one unit over this block's slice of d_in, then the block's partial is made available
@@ -515,11 +381,11 @@ __device__ __forceinline__ void shrink_unit(const FusedParams &P, const Unit &un
     constexpr int CW = 4096 / RP;      // columns per job
     constexpr int PW = TOK_PITCH;      // row pitch of the token rows
     // the four warps split the rank tiles WN ways and the chunk's columns WK ways, so that every
-    // warp owns two rank tiles of 8 and 64 columns of every job, whatever the bucket
+    // warp owns two rank tiles of 8 and 64 columns of every job (one column block), whatever the bucket
     constexpr int WN = RP / 16, WK = 4 / WN;
-    constexpr int KW = CW / WK;        // = 64 columns per warp and job
     constexpr int mrows = 8 * H;
     constexpr bool hi_rows = H == 2;
+    static_assert(CW / WK == 64, "a warp's share of a job is one block of 64 columns");
 
     unsigned char *smem = cx.smem;
     float *part = reinterpret_cast<float *>(smem + P.off_part);     // [WK][mrows][RP] = mrows x 64 floats
@@ -531,35 +397,57 @@ __device__ __forceinline__ void shrink_unit(const FusedParams &P, const Unit &un
     // chunks of a row exchanged by the row number's low three bits (128-byte swizzle).
     const uint32_t blk_bytes = (uint32_t)un.rb * 128u;
 
-    // warp (wk, wn) takes columns [wk*KW, (wk+1)*KW) of every chunk and rank tiles 2wn, 2wn+1
+    // warp (wk, wn) takes column block wk of every chunk and rank tiles 2wn, 2wn+1
     const int wk = warp % WK, wn = warp / WK;
+    // Operand fragments come by ldmatrix.  Lane l names row (l & 7) of 8x8 matrix (l >> 3).
+    //  weights: matrices (tile 2wn, k 0-7) (tile 2wn, k 8-15) (tile 2wn+1, k 0-7) (tile 2wn+1, k 8-15);
+    //           rank row n = 16 wn + 8 (mi >> 1) + r sits at n * 128 bytes of the column block, its
+    //           16-byte chunk c at ((c ^ r) << 4); c = 2 (ks / 16) + (mi & 1), whose even part is
+    //           folded in per step with one XOR
+    //  tokens:  matrices (rows 0-7, k 0-7) (rows 8-15, k 0-7) (rows 0-7, k 8-15) (rows 8-15, k 8-15)
+    const int mi = lane >> 3, r = lane & 7;
+    const uint32_t w_lane = (uint32_t)(16 * wn + 8 * (mi >> 1) + r) * 128u + (uint32_t)(((mi & 1) ^ r) << 4);
+    const uint32_t x_lane = hi_rows ? (uint32_t)(((mi & 1) * 8 + r) * PW + (mi >> 1) * 8) * 2u
+                                    : (uint32_t)(r * PW + (mi & 1) * 8) * 2u;
     float acc[2][4];
 #pragma unroll
     for (int i = 0; i < 2; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.0f;
     for (int32_t c = 0; c < un.na; ++c) {
         const int st = acquire_job(P, cx);
-        const unsigned char *As = smem + P.off_w + st * W_BYTES;   // tile of A_i
-        const __nv_bfloat16 *X = reinterpret_cast<const __nv_bfloat16 *>(smem + P.off_tok + st * P.tok_bytes);
-        const int32_t ncols = min(CW, un.a_hi - (un.a_lo + c * CW));
-        if (cx.ok) {
+        const uint32_t As = smem_u32(smem + P.off_w + st * W_BYTES) + (uint32_t)wk * blk_bytes + w_lane;
+        const uint32_t X = smem_u32(smem + P.off_tok + st * P.tok_bytes) + (uint32_t)(wk * 64 * 2) + x_lane;
+        const int32_t ncols = min(CW, un.a_hi - (un.a_lo + c * CW)) - wk * 64;   // of this warp's block
+        if (cx.ok && ncols >= 64) {
 #pragma unroll
-            for (int ks = 0; ks < KW; ks += 16) {
-                const int kk = wk * KW + ks;
-                if (kk < ncols) {
-                    const bool full = ncols - kk >= 16;   // else only 8 columns are left
-                    uint32_t a[4];
-                    a[0] = lds32(X + g * PW + kk + 2 * t);
-                    a[1] = hi_rows ? lds32(X + (g + 8) * PW + kk + 2 * t) : 0u;
-                    a[2] = full ? lds32(X + g * PW + kk + 8 + 2 * t) : 0u;
-                    a[3] = (full && hi_rows) ? lds32(X + (g + 8) * PW + kk + 8 + 2 * t) : 0u;
-                    const unsigned char *ab = As + (uint32_t)(kk >> 6) * blk_bytes + g * 128 + 4 * t;
-                    const uint32_t ch = (uint32_t)(kk & 63) >> 3;   // even
+            for (int ks = 0; ks < 64; ks += 16) {
+                uint32_t a[4], bw[4];
+                if (hi_rows) {
+                    ldmatrix_x4(a, X + ks * 2);
+                } else {
+                    ldmatrix_x2(a[0], a[2], X + ks * 2);
+                    a[1] = a[3] = 0u;
+                }
+                ldmatrix_x4(bw, As ^ (uint32_t)((ks >> 3) << 4));
+                mma16816(acc[0], a, bw[0], bw[1]);
+                mma16816(acc[1], a, bw[2], bw[3]);
+            }
+        } else if (cx.ok && ncols > 0) {
+            // ragged end of the slice: columns past the end hold neither x nor this adapter's weights
 #pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        const int nt = wn * 2 + i;
-                        mma16816(acc[i], a, lds32b(ab + nt * 1024 + ((ch ^ (uint32_t)g) << 4)),
-                                 full ? lds32b(ab + nt * 1024 + (((ch + 1) ^ (uint32_t)g) << 4)) : 0u);
+            for (int ks = 0; ks < 64; ks += 16) {
+                if (ks < ncols) {
+                    const bool full = ncols - ks >= 16;   // else only 8 columns are left
+                    uint32_t a[4], bw[4];
+                    if (hi_rows) {
+                        ldmatrix_x4(a, X + ks * 2);
+                    } else {
+                        ldmatrix_x2(a[0], a[2], X + ks * 2);
+                        a[1] = a[3] = 0u;
                     }
+                    ldmatrix_x4(bw, As ^ (uint32_t)((ks >> 3) << 4));
+                    if (!full) a[2] = a[3] = bw[1] = bw[3] = 0u;
+                    mma16816(acc[0], a, bw[0], bw[1]);
+                    mma16816(acc[1], a, bw[2], bw[3]);
                 }
             }
         }
@@ -586,8 +474,8 @@ __device__ __forceinline__ void shrink_unit(const FusedParams &P, const Unit &un
     // block partial: the column splits' sums in order
     if (cx.ok) {
         for (int i = tid; i < mrows * RP; i += FT) {
-            const int r = i / RP;
-            if (r < rows) {
+            const int rr = i / RP;
+            if (rr < rows) {
                 float v = part[i];
 #pragma unroll
                 for (int w = 1; w < WK; ++w) v += part[w * mrows * RP + i];
@@ -613,12 +501,13 @@ __device__ __forceinline__ void shrink_unit(const FusedParams &P, const Unit &un
 // then the expand over this block's slice of d_out with the fused epilogue.
 template <int RP, int H>
 __device__ __forceinline__ void expand_unit(const FusedParams &P, const Unit &un, const int32_t *rowidx,
-                                            Ctx &cx) {
+                                         Ctx &cx) {
     constexpr int CW = 4096 / RP;      // columns per job
     constexpr int PW = TOK_PITCH;
     constexpr int PV = RP + 8;         // pitch of the bf16 copies of v
     constexpr int NW = CW / 4;         // columns per warp and job
     constexpr int NT_E = NW / 8;       // column tiles of 8 per warp
+    constexpr int KT = RP / 16;        // k steps of 16 ranks the bucket can have
     constexpr int mrows = 8 * H;
     constexpr bool hi_rows = H == 2;
 
@@ -669,72 +558,101 @@ __device__ __forceinline__ void expand_unit(const FusedParams &P, const Unit &un
     ++cx.kr;
 
     // ---- expand: warp w takes columns [w*NW, (w+1)*NW) of every chunk ---------------------------
+    // v as MMA row operand, high and low parts; for the smallest bucket (one step of 16 ranks) the
+    // fragments stay in registers for all of the unit's jobs
+    uint32_t ah[KT == 1 ? 4 : 1], al[KT == 1 ? 4 : 1];
+    const __nv_bfloat16 *vh = Vh + g * PV + 2 * t;
+    const __nv_bfloat16 *vl = Vl + g * PV + 2 * t;
+    if (KT == 1) {
+        ah[0] = lds32(vh);
+        ah[1] = hi_rows ? lds32(vh + 8 * PV) : 0u;
+        ah[2] = lds32(vh + 8);
+        ah[3] = hi_rows ? lds32(vh + 8 * PV + 8) : 0u;
+        al[0] = lds32(vl);
+        al[1] = hi_rows ? lds32(vl + 8 * PV) : 0u;
+        al[2] = lds32(vl + 8);
+        al[3] = hi_rows ? lds32(vl + 8 * PV + 8) : 0u;
+    }
+    // B_i fragments by ldmatrix (transposing): lane l names rank row ks + 8 (mi & 1) + r of column
+    // tile 2 np + (mi >> 1); the tile's 16-byte chunk c sits at ((c ^ r) << 4), the even part of c
+    // is folded in per tile pair with one XOR
+    const int mi = lane >> 3, r = lane & 7;
+    const uint32_t b_lane = (uint32_t)((mi & 1) * 8 + r) * 128u + (uint32_t)(((mi >> 1) ^ r) << 4);
+    // this lane's output rows: g (and g + 8), columns 2t, 2t+1 of every column tile
+    const bool row0 = g < rows, row1 = hi_rows && g + 8 < rows;
+    __nv_bfloat16 *y0p = it.y + (int64_t)(row0 ? rowidx[g] : 0) * it.ldy + un.b_lo + warp * NW + 2 * t;
+    __nv_bfloat16 *y1p = it.y + (int64_t)(row1 ? rowidx[g + 8] : 0) * it.ldy + un.b_lo + warp * NW + 2 * t;
+    const uint32_t ys_lane = (uint32_t)(g * PW + warp * NW + 2 * t) * 2u;
     const float s = un.scale;
+    // the column block of this warp's first tile and the tile's chunk number inside it
+    constexpr int TPB = 8;   // column tiles per 64-column block
     for (int32_t c = 0; c < un.nb; ++c) {
         const int st = acquire_job(P, cx);
-        const unsigned char *Bs = smem + P.off_w + st * W_BYTES;   // tile of B_i
-        const __nv_bfloat16 *Ys = reinterpret_cast<const __nv_bfloat16 *>(smem + P.off_tok + st * P.tok_bytes);
-        const int32_t col0 = un.b_lo + c * CW, ncols = min(CW, un.b_hi - col0);
-        const int base = warp * NW;
-        // column tiles in groups of at most four: 16 accumulator registers at a time
-        constexpr int NG = NT_E < 4 ? NT_E : 4;
-        if (cx.ok) {
+        const uint32_t Bs = smem_u32(smem + P.off_w + st * W_BYTES) + b_lane;
+        const uint32_t Ys = smem_u32(smem + P.off_tok + st * P.tok_bytes) + ys_lane;
+        const int32_t ncols = min(CW, un.b_hi - (un.b_lo + c * CW)) - warp * NW;   // of this warp's columns
+        if (cx.ok && ncols > 0) {
 #pragma unroll
-            for (int j0 = 0; j0 < NT_E; j0 += NG) {
-                const int gbase = base + j0 * 8;
-                if (gbase >= ncols) break;
-                float ex[NG][4];
+            for (int np = 0; np < NT_E / 2; ++np) {
+                // tiles 2np, 2np+1 of this warp: columns warp*NW + 16 np .. + 15 of the chunk
+                if (NT_E > 2 && 16 * np >= ncols) break;
+                const int tile0 = 0;   // (placeholder for readability: tile index inside the warp's columns is 2 np)
+                (void)tile0;
+                float ex[2][4];
 #pragma unroll
-                for (int j = 0; j < NG; ++j) ex[j][0] = ex[j][1] = ex[j][2] = ex[j][3] = 0.0f;
-                const __nv_bfloat16 *vh = Vh + g * PV + 2 * t;
-                const __nv_bfloat16 *vl = Vl + g * PV + 2 * t;
-                for (int ks = 0; ks < rank16; ks += 16) {
-                    uint32_t ah[4], al[4];
-                    ah[0] = lds32(vh + ks);
-                    ah[1] = hi_rows ? lds32(vh + 8 * PV + ks) : 0u;
-                    ah[2] = lds32(vh + ks + 8);
-                    ah[3] = hi_rows ? lds32(vh + 8 * PV + ks + 8) : 0u;
-                    al[0] = lds32(vl + ks);
-                    al[1] = hi_rows ? lds32(vl + 8 * PV + ks) : 0u;
-                    al[2] = lds32(vl + ks + 8);
-                    al[3] = hi_rows ? lds32(vl + 8 * PV + ks + 8) : 0u;
+                for (int j = 0; j < 2; ++j) ex[j][0] = ex[j][1] = ex[j][2] = ex[j][3] = 0.0f;
+                // absolute tile number in the chunk: warp * NT_E + 2 np; its column block and chunk
+                const uint32_t tabs = (uint32_t)(warp * NT_E + 2 * np);
+                const uint32_t baddr = Bs + (tabs / TPB) * blk_bytes;
+                const uint32_t cx4 = (tabs % TPB) << 4;
+#pragma unroll
+                for (int kt = 0; kt < KT; ++kt) {
+                    const int ks = kt * 16;
+                    if (KT > 1 && ks >= rank16) break;
+                    uint32_t fh[4], fl[4];
+                    if (KT == 1) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) { fh[q] = ah[q]; fl[q] = al[q]; }
+                    } else {
+                        fh[0] = lds32(vh + ks);
+                        fh[1] = hi_rows ? lds32(vh + 8 * PV + ks) : 0u;
+                        fh[2] = lds32(vh + ks + 8);
+                        fh[3] = hi_rows ? lds32(vh + 8 * PV + ks + 8) : 0u;
+                        fl[0] = lds32(vl + ks);
+                        fl[1] = hi_rows ? lds32(vl + 8 * PV + ks) : 0u;
+                        fl[2] = lds32(vl + ks + 8);
+                        fl[3] = hi_rows ? lds32(vl + 8 * PV + ks + 8) : 0u;
+                    }
+                    uint32_t bb[4];
+                    ldmatrix_x4_trans(bb, (baddr + (uint32_t)ks * 128u) ^ cx4);
                     // Rank rows ks+8 .. ks+15 were only copied when the tile has them; what the
                     // stage holds there otherwise belongs to an earlier job (possibly another
                     // adapter's weights) and must not meet the MMA, not even multiplied by zero.
-                    const bool upper = ks + 8 < un.rb;
-#pragma unroll
-                    for (int np = 0; np < NG / 2; ++np) {
-                        // matrices: (k 0..7, tile 2np), (k 8..15, tile 2np), (k 0..7, 2np+1), (k 8..15, 2np+1)
-                        const int mi = lane >> 3;
-                        const int col = gbase + (np * 2 + (mi >> 1)) * 8;
-                        const unsigned char *bp = Bs + (uint32_t)(col >> 6) * blk_bytes +
-                                                  (ks + (mi & 1) * 8 + (lane & 7)) * 128 +
-                                                  ((((uint32_t)(col & 63) >> 3) ^ (uint32_t)(lane & 7)) << 4);
-                        uint32_t bb[4];
-                        ldmatrix_x4_trans(bb, smem_u32(bp));
-                        if (!upper) bb[1] = bb[3] = 0u;
-                        mma16816(ex[np * 2], ah, bb[0], bb[1]);
-                        mma16816(ex[np * 2], al, bb[0], bb[1]);
-                        mma16816(ex[np * 2 + 1], ah, bb[2], bb[3]);
-                        mma16816(ex[np * 2 + 1], al, bb[2], bb[3]);
-                    }
+                    if (ks + 8 >= un.rb) bb[1] = bb[3] = 0u;
+                    mma16816(ex[0], fh, bb[0], bb[1]);
+                    mma16816(ex[0], fl, bb[0], bb[1]);
+                    mma16816(ex[1], fh, bb[2], bb[3]);
+                    mma16816(ex[1], fl, bb[2], bb[3]);
                 }
                 // epilogue straight from the accumulator layout: each lane owns two adjacent columns of
                 // a row per column tile; a quad covers 16 contiguous bytes
 #pragma unroll
-                for (int h = 0; h < H; ++h) {
-                    const int32_t m = g + 8 * h;
-                    if (m < rows) {
-                        __nv_bfloat16 *yrow = it.y + (int64_t)rowidx[m] * it.ldy + col0 + gbase + 2 * t;
-                        const __nv_bfloat16 *ybrow = Ys + m * PW + gbase + 2 * t;
-#pragma unroll
-                        for (int j = 0; j < NG; ++j) {
-                            if (gbase + j * 8 < ncols) {
-                                const uint32_t w = lds32(ybrow + j * 8);
-                                const float y0 = fmaf(s, ex[j][2 * h], __uint_as_float(w << 16));
-                                const float y1 = fmaf(s, ex[j][2 * h + 1], __uint_as_float(w & 0xffff0000u));
-                                *reinterpret_cast<uint32_t *>(yrow + j * 8) = pack2(y0, y1);
-                            }
+                for (int j = 0; j < 2; ++j) {
+                    const int coff = (2 * np + j) * 8;   // column offset inside the warp's columns
+                    if (coff < ncols) {
+                        if (row0) {
+                            uint32_t w;
+                            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w) : "r"(Ys + coff * 2));
+                            const float a0 = fmaf(s, ex[j][0], __uint_as_float(w << 16));
+                            const float a1 = fmaf(s, ex[j][1], __uint_as_float(w & 0xffff0000u));
+                            *reinterpret_cast<uint32_t *>(y0p + c * CW + coff) = pack2(a0, a1);
+                        }
+                        if (row1) {
+                            uint32_t w;
+                            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w) : "r"(Ys + (8 * PW + coff) * 2));
+                            const float a0 = fmaf(s, ex[j][2], __uint_as_float(w << 16));
+                            const float a1 = fmaf(s, ex[j][3], __uint_as_float(w & 0xffff0000u));
+                            *reinterpret_cast<uint32_t *>(y1p + c * CW + coff) = pack2(a0, a1);
                         }
                     }
                 }
@@ -775,54 +693,56 @@ template <int H>
 __device__ __forceinline__ void consumer_warps(const FusedParams &P, Ctx &cx) {
     unsigned char *smem = cx.smem;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    Walk w;
     {
-        // the number of units and the records of this cluster's first two units, side by side
-        int32_t n_units = P.meta ? ldg_int(P.meta + H_NPIECE) : P.T;
+        // the number of units and (speculatively, as if the table were full) the records of this
+        // cluster's first two units, side by side
+        const int32_t n_hdr = P.meta ? ldg_int(P.meta + H_NPIECE) : P.T;
         UnitRegs m0, m1;
+        const bool spec = P.n_items == 1;
         if (warp == 3) {
-            m0 = fetch_unit(P, cx.cid, P.units_cap, P.units_cap * P.n_items, lane);
-            m1 = fetch_unit(P, cx.cid + cx.G, P.units_cap, P.units_cap * P.n_items, lane);
+            m0 = fetch_unit(P, cx.cid, spec && cx.cid < P.units_cap, lane);
+            m1 = fetch_unit(P, cx.cid + cx.G, spec && cx.cid + cx.G < P.units_cap, lane);
         }
-        if (n_units > P.units_cap) n_units = P.units_cap;
-        cx.total = n_units * P.n_items;
-        if (n_units < 1) n_units = 1;
-        cx.n_units = n_units;
+        set_counts(P, cx, n_hdr);
+        w.start(cx.cid, cx.n_units);
+        const Walk w1 = w.next(cx.G, cx.n_units);
         if (warp == 3) {
-            // the speculative fetch above used the capacity for the unit count: right when they
-            // agree (one projection, or a full table), else fetched again
-            if (n_units != P.units_cap && P.n_items > 1) {
-                m0 = fetch_unit(P, cx.cid, n_units, cx.total, lane);
-                m1 = fetch_unit(P, cx.cid + cx.G, n_units, cx.total, lane);
+            if (!spec) {
+                m0 = fetch_unit(P, w.u, w.g < cx.total, lane);
+                m1 = fetch_unit(P, w1.u, w1.g < cx.total, lane);
             }
-            store_unit(smem, 0, m0, cx.cid < cx.total, lane);
-            store_unit(smem, 1, m1, cx.cid + cx.G < cx.total, lane);
+            store_unit(smem, 0, m0, w.g < cx.total, lane);
+            store_unit(smem, 1, m1, w1.g < cx.total, lane);
         }
     }
     consumer_sync();
     if (P.early) griddep_wait();
 
-    int32_t pend_i = -1;   // iteration whose unit still has its expand half to run
-    auto entry_of = [&](int32_t i) { return smem + SM_RING + (i % UNIT_RING) * RING_ENTRY; };
+    // the unit whose expand half is still to run: its ring entry and projection
+    int32_t pend_i = -1, pend_item = 0;
+    auto entry_of = [&](int32_t i) { return smem + SM_RING + (i & (UNIT_RING - 1)) * RING_ENTRY; };
     auto run_pending = [&]() {
         if (pend_i < 0) return;
         const unsigned char *e = entry_of(pend_i);
-        const Unit up = decode_unit(P, cx, *reinterpret_cast<const int4 *>(e), cx.cid + pend_i * cx.G);
+        const Unit up = decode_unit(P, cx, *reinterpret_cast<const int4 *>(e), pend_item);
         expand_dispatch<H>(P, up, reinterpret_cast<const int32_t *>(e + 16), cx);
         pend_i = -1;
     };
-    for (int32_t i = 0;; ++i) {
-        const int32_t g = cx.cid + i * cx.G;
-        if (g >= cx.total) break;
+    Walk w1 = w.next(cx.G, cx.n_units);
+    for (int32_t i = 0; w.g < cx.total; ++i) {
         // the record of the unit after next is requested now and stored when this step is done
+        const Walk w2 = w1.next(cx.G, cx.n_units);
         UnitRegs mn;
-        if (warp == 3) mn = fetch_unit(P, g + 2 * cx.G, cx.n_units, cx.total, lane);
+        if (warp == 3) mn = fetch_unit(P, w2.u, w2.g < cx.total, lane);
         const unsigned char *e = entry_of(i);
         const int4 rec = *reinterpret_cast<const int4 *>(e);
-        const Unit un = decode_unit(P, cx, rec, g);
+        const Unit un = decode_unit(P, cx, rec, w.item);
         if (un.run) shrink_dispatch<H>(P, un, cx);
         run_pending();
         if (un.run) {
             pend_i = i;
+            pend_item = w.item;
         } else if (!P.meta && rec.x == -1) {   // per-token mode: this token has no adapter
             if (cx.crank == 0 && tid == 0 && rec.y && un.item == 0)
                 atomicAdd(&P.pool.status[STATUS_INVALID_TOKENS], 1);
@@ -832,6 +752,8 @@ __device__ __forceinline__ void consumer_warps(const FusedParams &P, Ctx &cx) {
         }
         if (warp == 3) store_unit(smem, i + 2, mn, true, lane);
         consumer_sync();   // the new record is visible; nobody reads the overwritten one any more
+        w = w1;
+        w1 = w2;
     }
     run_pending();
     if (!cx.ok) {
@@ -844,8 +766,8 @@ __device__ __forceinline__ void consumer_warps(const FusedParams &P, Ctx &cx) {
         int32_t *rowidx = reinterpret_cast<int32_t *>(smem + SM_RING + 16);
         const int32_t n_idle = P.T - __ldg(P.meta + H_NACTIVE);
         const int32_t chunks = (n_idle + 15) / 16;
-        for (int32_t w = cx.cid; w < chunks * P.n_items; w += cx.G) {
-            const int32_t item = w / chunks, first = (w - item * chunks) * 16;
+        for (int32_t k = cx.cid; k < chunks * P.n_items; k += cx.G) {
+            const int32_t item = k / chunks, first = (k - item * chunks) * 16;
             if (P.item[item].in_place) continue;
             const int32_t rows = min(16, n_idle - first);
             consumer_sync();
@@ -869,8 +791,11 @@ fused_kernel(const __grid_constant__ FusedParams P) {
     cx.crank = cluster_ctarank();
     cx.cid = (int32_t)(blockIdx.x / cx.csize);
     cx.G = (int32_t)(gridDim.x / cx.csize);
-    cx.cq = cx.kp = cx.kr = 0;
-    cx.n_units = cx.total = 0;
+    cx.st = 0;
+    cx.ph = 0;
+    cx.kp = cx.kr = 0;
+    cx.n_units = 1;
+    cx.total = 0;
     cx.ok = true;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // The next kernel of the stream may become resident from now on.  It touches nothing this
@@ -916,7 +841,7 @@ fused_kernel(const __grid_constant__ FusedParams P) {
     __syncthreads();
     if (*dead_flag(smem) && tid == 0) {
         const int32_t issued = *reinterpret_cast<volatile int32_t *>(smem + SM_ISSUED);
-        // stages of jobs that were requested but whose data nobody waited for
+        // the most recent job of every stage: all earlier ones were waited for before a refill
         for (int32_t q = max(issued - P.n_stages, 0); q < issued; ++q)
             mbar_wait(&cx.full[q % P.n_stages], (uint32_t)(q / P.n_stages) & 1u);
     }
@@ -926,6 +851,12 @@ fused_kernel(const __grid_constant__ FusedParams P) {
     cluster_arrive();
     cluster_wait();
 }
+
+}  // namespace lora
+
+#include "decode_kernel.cuh"
+
+namespace lora {
 
 // ---------------------------------------------------------------------------------------------
 // host side: tensor maps (built once per pool, kept in the pool's device buffer) and launch
@@ -987,12 +918,15 @@ lora_status_t build_fused_maps(lora_pool_t *pool) {
 }
 
 // Shared-memory carve-up and launch.  The buffers are sized for the largest rank bucket that has
-// ever been loaded into the pool.
+// ever been loaded into the pool.  H = 0: the decode kernel (its own fixed carve-up).
 template <int H>
 static lora_status_t launch_h(lora_pool_t *pool, FusedParams &P, int32_t C, const void *meta_key,
                               cudaStream_t stream) {
-    auto kern = fused_kernel<H>;
-    const int32_t mrows = 8 * H;
+    void (*kern)(const FusedParams) = nullptr;
+    if (H == 0) kern = decode_kernel;
+    else if (H == 1) kern = fused_kernel<1>;
+    else kern = fused_kernel<2>;
+    const int32_t mrows = H == 2 ? 16 : 8;
     const int32_t RPmax = (pool->bucket_mask & 8u) ? 64 : (pool->bucket_mask & 4u) ? 32 : 16;
     int32_t S = pool->tuning[5];
     if (S < 2 || S > MAX_STAGES) S = 2;   // two stages and more resident blocks beat deeper rings
@@ -1010,10 +944,10 @@ static lora_status_t launch_h(lora_pool_t *pool, FusedParams &P, int32_t C, cons
     P.tok_bytes = mrows * TOK_PITCH * 2;
     P.off_tok = o;    o += S * P.tok_bytes;
     P.n_stages = S;
-    const int32_t smem = o;
+    const int32_t smem = H == 0 ? dec::smem_bytes(S) : o;
     P.prefetch = pool->tuning[8] == 1 ? 0 : 1;
 
-    lora_pool::FusedLaunchCache &lc = pool->fused_cache[H - 1];
+    lora_pool::FusedLaunchCache &lc = pool->fused_cache[H];
     if (smem > lc.attr_smem) {
         LORA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         lc.attr_smem = smem;
@@ -1121,6 +1055,17 @@ lora_status_t launch_fused_items(lora_pool_t *pool, const ApplyParams *items, in
         it.map_base = target * MAPS_PER_TARGET;
         it.in_place = A.in_place;
     }
+    // Decode batches take the decode kernel: grouped metadata with units of at most 8 rows, no
+    // adapter above rank 16 in the pool, widths in whole 64-column blocks and no block of the
+    // cluster without columns (tuning key 10 = 1: always the general kernel).
+    bool decode = A0.meta && tile_m <= 8 && (pool->bucket_mask & 12u) == 0 && P.path_filter == 0 &&
+                  pool->tuning[10] != 1;
+    for (int32_t i = 0; i < n_items && decode; ++i) {
+        const FusedItem &it = P.item[i];
+        decode = it.d_in % 64 == 0 && it.d_out % 64 == 0 && (C - 1) * it.wa < it.d_in &&
+                 (C - 1) * it.wb < it.d_out;
+    }
+    if (decode) return launch_h<0>(pool, P, C, A0.meta, stream);
     return tile_m <= 8 ? launch_h<1>(pool, P, C, A0.meta, stream) : launch_h<2>(pool, P, C, A0.meta, stream);
 }
 

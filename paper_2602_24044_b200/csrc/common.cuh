@@ -147,7 +147,7 @@ struct lora_pool {
     struct FusedLaunchCache {
         int32_t attr_smem = 0, occ_smem = 0, occ_c = 0, occ_clusters = 0;
     };
-    FusedLaunchCache fused_cache[2];
+    FusedLaunchCache fused_cache[3];
 
     // Shapes of the metadata tables built through this handle (the table itself lives on the
     // device; apply calls need T and tile_m on the host to size their grids).
