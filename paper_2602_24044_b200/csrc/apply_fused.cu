@@ -85,6 +85,8 @@ struct FusedParams {
     int32_t push;              // block partials are pushed to all blocks of the cluster (small units)
     int32_t path_filter;       // 0 = every unit; else skip runs of at least this many consecutive tokens
     int32_t prefetch;          // ask L2 for the next unit's tiles and rows ahead of the ring
+    int32_t late_trigger;      // decode kernel: let the successor in only once this kernel's blocks are set up
+    int32_t copy_idle;         // some projection is out of place: rows without adapter are copied
     int32_t off_part, off_vpart, vbuf_bytes, off_vh, off_vl;   // warp partials, exchange buffers (x2), v as bf16 high / low parts
     int32_t off_w, off_tok, tok_bytes, n_stages;               // ring of job buffers: weight tiles, token rows
     int32_t moff_perm, moff_udesc, moff_uperm;                 // word offsets: perm, unit records, unit row ids
@@ -946,6 +948,9 @@ static lora_status_t launch_h(lora_pool_t *pool, FusedParams &P, int32_t C, cons
     P.n_stages = S;
     const int32_t smem = H == 0 ? dec::smem_bytes(S) : o;
     P.prefetch = pool->tuning[8] == 1 ? 0 : 1;
+    P.late_trigger = pool->tuning[11] == 1 ? 1 : 0;
+    P.copy_idle = 0;
+    for (int32_t i = 0; i < P.n_items; ++i) P.copy_idle |= P.item[i].in_place ? 0 : 1;
 
     lora_pool::FusedLaunchCache &lc = pool->fused_cache[H];
     if (smem > lc.attr_smem) {

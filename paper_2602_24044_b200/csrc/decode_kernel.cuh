@@ -105,35 +105,35 @@ __device__ __forceinline__ void p_request(const FusedParams &P, unsigned char *s
     }
 }
 
-// L2 hints for a unit: its weight tiles from job `first` on and the block's slices of its rows.
-__device__ __forceinline__ void p_hint(const FusedParams &P, const PUnit &un, int32_t first, int32_t rowid,
-                                       int lane) {
-    if (!un.run) return;
-    const FusedItem &it = P.item[un.item];
-    const CUtensorMap *ma = P.maps + it.map_base + (un.rb >> 3) - 1;
-    for (int32_t j = first + lane; j < un.na + un.nb; j += 32) {
-        const bool shrink = j < un.na;
-        const int32_t col0 = shrink ? un.a_lo + j * 256 : un.b_lo + (j - un.na) * 256;
-        tma_prefetch_4d(shrink ? ma : ma + 8, 0, 0, col0 >> 6, un.slot);
+// The first global loads of the requesting warp: the unit count and (speculatively, as if the
+// table were full) the cluster's first record, side by side.  Issued at the very top of the kernel
+// when the table may be read ahead of the preceding kernel's end, else after the wait.
+struct FirstLoads {
+    int32_t n_units;
+    int4 rec;
+    int32_t rowid;
+};
+__device__ __forceinline__ FirstLoads first_loads(const FusedParams &P, int32_t cid, int lane) {
+    FirstLoads f;
+    f.n_units = ldg_int(P.meta + H_NPIECE);
+    f.rec = make_int4(-2, 0, 0, 0);
+    f.rowid = 0;
+    if (P.n_items == 1 && cid < P.units_cap) {
+        if (lane == 16) f.rec = ldg_int4(P.meta + P.moff_udesc + 4 * (int64_t)cid);
+        else if (lane < 16) f.rowid = ldg_int(P.meta + P.moff_uperm + 16 * (int64_t)cid + lane);
     }
-    if (lane < un.rows) {
-        if (un.a_hi > un.a_lo)
-            bulk_prefetch_l2(it.x + (int64_t)rowid * it.ldx + un.a_lo, (uint32_t)(un.a_hi - un.a_lo) * 2u);
-        if (un.b_hi > un.b_lo)
-            bulk_prefetch_l2(it.yb + (int64_t)rowid * it.ldyb + un.b_lo, (uint32_t)(un.b_hi - un.b_lo) * 2u);
-    }
+    return f;
 }
 
 __device__ __forceinline__ void producer(const FusedParams &P, unsigned char *smem, int32_t cid, int32_t G,
-                                         uint32_t crank, int lane) {
+                                         uint32_t crank, int lane, const FirstLoads &fl) {
     const int32_t S = P.n_stages;
     volatile int32_t *dead = reinterpret_cast<volatile int32_t *>(smem + SM_FLAG);
     volatile int32_t *count = reinterpret_cast<volatile int32_t *>(smem + SM_COUNT);
     uint64_t *empty = reinterpret_cast<uint64_t *>(smem + SM_EMPTY);
-    // the unit count and (speculatively, as if the table were full) the first record, side by side
-    int32_t n_units = ldg_int(P.meta + H_NPIECE);
-    int4 rec = make_int4(-2, 0, 0, 0);
-    int32_t rowid = 0;
+    int32_t n_units = fl.n_units;
+    int4 rec = fl.rec;
+    int32_t rowid = fl.rowid;
     auto fetch = [&](int32_t u, bool valid, int4 &r, int32_t &id) {
         r = make_int4(-2, 0, 0, 0);
         id = 0;
@@ -149,7 +149,6 @@ __device__ __forceinline__ void producer(const FusedParams &P, unsigned char *sm
         r.w = __shfl_sync(0xffffffffu, r.w, 16);
         return r;
     };
-    if (P.n_items == 1) fetch(cid, cid < P.units_cap, rec, rowid);
     if (n_units > P.units_cap) n_units = P.units_cap;
     const int32_t total = n_units * P.n_items;
     if (n_units < 1) n_units = 1;
@@ -191,18 +190,11 @@ __device__ __forceinline__ void producer(const FusedParams &P, unsigned char *sm
             if (P.early) {
                 // The kernel before this one may still be running: the pool may be read (the host
                 // vouches for it), the activations not yet.  Weight tiles of the first jobs now, their
-                // token rows after the wait; everything else of this and the next unit as L2 hints.
+                // token rows after the wait.
                 skip = !un.run ? 0 : un.na < S ? un.na : S;
                 for (int32_t j = 0; j < skip; ++j) p_request(P, smem, un, j, entry, j, rowid, lane, 1);
             }
-            if (P.prefetch) p_hint(P, un, skip, rowid, lane);
         }
-        const bool hint_next = P.prefetch && next_real;
-        const bool hint_first = i == 0 && !waited;   // time to spare before the wait returns
-        PUnit un_next;
-        un_next.run = false;
-        if (hint_next) un_next = p_decode(P, crank, bcast(rec_n), itn);
-        if (hint_next && hint_first) p_hint(P, un_next, 0, rowid_n, lane);
         if (!waited) {
             griddep_wait();
             waited = true;
@@ -216,7 +208,6 @@ __device__ __forceinline__ void producer(const FusedParams &P, unsigned char *sm
         // this step's jobs in ring order: the unit's shrink chunks, then the pending unit's expand chunks
         const int32_t ja = un.run ? un.na : 0, jb = have_pend ? pend.nb : 0;
         for (int32_t k = (i == 0 ? skip : 0); k < ja + jb; ++k) {
-            if (k == ja && hint_next && !hint_first) p_hint(P, un_next, 0, rowid_n, lane);
             if (q >= S && ok) {
                 ok = mbar_wait(&empty[st], (ph - 1u) & 1u);
                 if (!ok) *dead = 1;
@@ -229,7 +220,6 @@ __device__ __forceinline__ void producer(const FusedParams &P, unsigned char *sm
             ++q;
             if (++st == S) { st = 0; ++ph; }
         }
-        if (jb == 0 && hint_next && !hint_first) p_hint(P, un_next, 0, rowid_n, lane);
         have_pend = un.run;
         pend = un;
         pend_rowid = rowid;
@@ -286,6 +276,9 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
     int32_t st = 0, kp = 0, kr = 0;
     uint32_t ph = 0, blk_bytes = 0;
     bool ok = true;
+    bool met_cluster = false;   // the opening cluster barrier has been waited for (needed before the first remote access)
+    // rows without adapter are copied at the end (out-of-place projections): their number, asked for now
+    const int32_t n_active = P.copy_idle ? ldg_int(P.meta + H_NACTIVE) : P.T;
     // The consumer threads meet on an mbarrier, not on bar.sync: a thread that has given up a wait
     // never arrives, and the others must not wait for it without a limit.
     uint32_t cs = 0;
@@ -343,17 +336,21 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
                 float *p0 = part + (warp * 8 + g) * 16 + 2 * t;
                 *reinterpret_cast<float2 *>(p0) = make_float2(acc[0][0], acc[0][1]);
                 *reinterpret_cast<float2 *>(p0 + 8) = make_float2(acc[1][0], acc[1][1]);
+                if (!met_cluster) {   // no block is written to before its barriers are set up
+                    cluster_wait();
+                    met_cluster = true;
+                }
+                // this block will receive rows x 16 floats from every block of the cluster
+                if (tid == 0) mbar_expect_tx(reinterpret_cast<uint64_t *>(smem + SM_XB) + b, csize * (uint32_t)rows * 64u);
                 if (!meet()) { ok = false; break; }
-                // thread (row, rank): the four column blocks' sums in order, pushed to every block
+                // thread (row, rank): the four column blocks' sums in order, sent to every block; each
+                // store counts its bytes on the receiver's barrier, so data and signal travel together
                 if ((tid >> 4) < rows) {
                     const float v = ((part[tid] + part[128 + tid]) + part[256 + tid]) + part[384 + tid];
                     const uint32_t dst = smem_u32(smem + SM_VALL + b * 4096 + ((int)crank * 128 + tid) * 4);
-                    for (uint32_t q = 0; q < csize; ++q) st_peer_f32(dst, q, v);
+                    const uint32_t bar = smem_u32(smem + SM_XB + 8 * b);
+                    for (uint32_t q = 0; q < csize; ++q) st_async_peer_f32(dst, bar, q, v);
                 }
-                // one arrival per block and peer: thread q tells block q, after the block's threads
-                // have met (its release then covers all their writes)
-                if (!meet()) { ok = false; break; }
-                if (tid < (int)csize) mbar_arrive_peer(reinterpret_cast<uint64_t *>(smem + SM_XB) + b, (uint32_t)tid);
                 ++kp;
             }
         } else {
@@ -451,11 +448,15 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
         }
     }
     if (!ok && tid == 0) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
+    // this block's last remote access is behind it: the closing cluster barrier is arrived at now
+    // and waited for at the very end of the kernel
+    if (!met_cluster) cluster_wait();
+    cluster_arrive();
 
     // rows that take no adapter: y_base -> y, 16 rows per cluster step (out-of-place projections)
-    if (ok && !*dead) {
+    if (ok && !*dead && n_active < P.T) {
         int32_t *rowidx = reinterpret_cast<int32_t *>(smem + SM_PART);
-        const int32_t n_idle = P.T - __ldg(P.meta + H_NACTIVE);
+        const int32_t n_idle = P.T - n_active;
         const int32_t chunks = (n_idle + 15) / 16;
         for (int32_t k = cid; k < chunks * P.n_items; k += G) {
             const int32_t item = k / chunks, first = (k - item * chunks) * 16;
@@ -487,7 +488,7 @@ decode_kernel(const __grid_constant__ FusedParams P) {
     // The next kernel of the stream may become resident from now on.  It touches nothing this
     // kernel writes before its own griddepcontrol.wait, which returns only when this kernel (and,
     // through this kernel's own wait below, everything before it) is complete.
-    griddep_launch_dependents();
+    if (!P.late_trigger) griddep_launch_dependents();
     // the swizzled tiles want 1024-byte aligned stages (the base is the same in every block, so
     // either all blocks of the launch leave here or none)
     if (smem_u32(smem) & 1023u) {
@@ -495,6 +496,14 @@ decode_kernel(const __grid_constant__ FusedParams P) {
         griddep_wait();
         return;
     }
+    // what the requesting warp needs first from global memory, asked for before anything else when
+    // the table may be read now
+    dec::FirstLoads fl;
+    fl.n_units = 0;
+    fl.rec = make_int4(-2, 0, 0, 0);
+    fl.rowid = 0;
+    if (warp == 4 && P.early) fl = dec::first_loads(P, cid, lane);
+    if (warp == 4 && lane < MAPS_PER_TARGET) prefetch_tensormap(P.maps + P.item[0].map_base + lane);
     if (tid == 0) {
         uint64_t *full = reinterpret_cast<uint64_t *>(smem + dec::SM_FULL);
         uint64_t *empty = reinterpret_cast<uint64_t *>(smem + dec::SM_EMPTY);
@@ -503,7 +512,7 @@ decode_kernel(const __grid_constant__ FusedParams P) {
             mbar_init(&empty[s], 4);
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(reinterpret_cast<uint64_t *>(smem + dec::SM_XB) + b, csize);
+            mbar_init(reinterpret_cast<uint64_t *>(smem + dec::SM_XB) + b, 1);
             mbar_init(reinterpret_cast<uint64_t *>(smem + dec::SM_YB) + b, 4 * csize);
         }
         mbar_init(reinterpret_cast<uint64_t *>(smem + dec::SM_CBAR), FT);
@@ -511,17 +520,23 @@ decode_kernel(const __grid_constant__ FusedParams P) {
         *reinterpret_cast<int32_t *>(smem + dec::SM_COUNT) = 0;
         fence_mbar_init();
     }
-    // no block signals a peer whose barriers are not set up
+    __syncthreads();
+    // opening cluster barrier: arrived at here, waited for only where a block first touches a peer
     cluster_arrive();
-    if (warp == 4 && lane < MAPS_PER_TARGET) prefetch_tensormap(P.maps + P.item[0].map_base + lane);
     // Activations are only touched after griddep_wait().  The unit records and the pool were
     // complete before the preceding kernel started when P.early is set (the host sets it only
     // then), so they are read, and the first weight tiles requested, ahead of the wait.
-    if (!P.early) griddep_wait();
-    __syncthreads();
-    cluster_wait();
-    if (warp == 4) dec::producer(P, smem, cid, G, crank, lane);
-    else dec::consumers(P, smem, cid, G, crank, csize);
+    if (!P.early) {
+        griddep_wait();
+        if (warp == 4) fl = dec::first_loads(P, cid, lane);
+    }
+    if (warp == 4) {
+        dec::producer(P, smem, cid, G, crank, lane, fl);
+        cluster_wait();     // the opening barrier (this warp touches no peer)
+        cluster_arrive();   // the closing one
+    } else {
+        dec::consumers(P, smem, cid, G, crank, csize);
+    }
     // A block that gave up may still have copies on their way into its shared memory; they must
     // land before the block leaves: all five warps meet, then one thread waits, bounded, for the
     // most recent job of every stage.
@@ -532,9 +547,9 @@ decode_kernel(const __grid_constant__ FusedParams P) {
             mbar_wait(reinterpret_cast<uint64_t *>(smem + dec::SM_FULL) + q % P.n_stages,
                       (uint32_t)(q / P.n_stages) & 1u);
     }
-    // No block leaves while a peer may still write into its buffers or signal its barriers: the
-    // closing barrier is the hardware one, which every block reaches whatever happened before.
-    cluster_arrive();
+    // No block leaves while a peer may still write into its buffers or signal its barriers: every
+    // block of the cluster has arrived at the closing barrier (the hardware one, which each block
+    // reaches whatever happened before) only after its last access to a peer.
     cluster_wait();
 }
 

@@ -116,6 +116,17 @@ __device__ __forceinline__ void st_peer_f32(uint32_t local_addr, uint32_t rank, 
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
     asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
 }
+// write a float at the same shared-memory offset in block `rank` of the cluster and count its four
+// bytes on the mbarrier at offset `local_bar` of that block: whoever sees the barrier's phase
+// complete also sees the data
+__device__ __forceinline__ void st_async_peer_f32(uint32_t local_addr, uint32_t local_bar, uint32_t rank, float v) {
+    uint32_t remote, rbar;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(local_bar), "r"(rank));
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(remote),
+                 "r"(__float_as_uint(v)), "r"(rbar)
+                 : "memory");
+}
 // D += A(16x16, row) . B(16x8, col), bf16 inputs, fp32 accumulate
 __device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
                                          uint32_t b1) {
