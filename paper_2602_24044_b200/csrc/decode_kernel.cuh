@@ -37,7 +37,7 @@ constexpr int SM_W = 11264;                      // weight tiles, W_BYTES per st
 constexpr int TOK_BYTES = 8 * TOK_PITCH * 2;     // token rows of a stage
 static_assert(SM_VALL + 2 * 4096 <= SM_W && SM_W % 1024 == 0, "header fits");
 
-enum { J_SHRINK = 1, J_FIRST = 2, J_LAST = 4, J_END = 8 };
+enum { J_SHRINK = 1, J_FIRST = 2, J_LAST = 4, J_END = 8 /* no data, stream over */, J_FINAL = 16 /* last job of the stream */ };
 
 struct UnitEntry {          // 64 bytes
     int32_t rows, rb, rank, item;
@@ -81,7 +81,8 @@ __device__ __forceinline__ PUnit p_decode(const FusedParams &P, uint32_t crank, 
 // One job into stage st: header, weight tile, token rows.  mode 0: all; 1: header and tile (with the
 // byte count of the whole job); 2: the token rows of a job started in mode 1.
 __device__ __forceinline__ void p_request(const FusedParams &P, unsigned char *smem, const PUnit &un,
-                                          int32_t j, int32_t entry, int st, int32_t rowid, int lane, int mode) {
+                                          int32_t j, int32_t entry, int st, int32_t rowid, int lane, int mode,
+                                          bool final_job = false) {
     const FusedItem &it = P.item[un.item];
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + SM_FULL) + st;
     const bool shrink = j < un.na;
@@ -91,7 +92,8 @@ __device__ __forceinline__ void p_request(const FusedParams &P, unsigned char *s
     if (lane == 0 && mode != 2) {
         const int32_t last = shrink ? un.na - 1 : un.nb - 1;
         *reinterpret_cast<int4 *>(smem + SM_JOB + 16 * st) =
-            make_int4((shrink ? J_SHRINK : 0) | (c == 0 ? J_FIRST : 0) | (c == last ? J_LAST : 0), entry, c, ncols);
+            make_int4((shrink ? J_SHRINK : 0) | (c == 0 ? J_FIRST : 0) | (c == last ? J_LAST : 0) |
+                          (final_job ? J_FINAL : 0), entry, c, ncols);
         const CUtensorMap *map = P.maps + it.map_base + (shrink ? 0 : 8) + (un.rb >> 3) - 1;
         // the tile load always delivers its whole box: rb rows of 256 columns
         mbar_expect_tx(full, (uint32_t)un.rb * 512u + (uint32_t)un.rows * (uint32_t)ncols * 2u);
@@ -162,6 +164,7 @@ __device__ __forceinline__ void producer(const FusedParams &P, unsigned char *sm
     bool ok = true, have_pend = false, waited = !P.early;
     PUnit pend;
     int32_t pend_rowid = 0, pend_entry = 0;
+    bool sent_final = false;
     for (int32_t i = 0;; ++i) {
         const bool real = g < total;
         if (!real && !have_pend) break;
@@ -193,6 +196,14 @@ __device__ __forceinline__ void producer(const FusedParams &P, unsigned char *sm
                 // token rows after the wait.
                 skip = !un.run ? 0 : un.na < S ? un.na : S;
                 for (int32_t j = 0; j < skip; ++j) p_request(P, smem, un, j, entry, j, rowid, lane, 1);
+                // and a hint to L2 for the block's slices of the unit's rows (no value is consumed)
+                if (un.run && lane < un.rows) {
+                    const FusedItem &it = P.item[un.item];
+                    if (un.a_hi > un.a_lo)
+                        bulk_prefetch_l2(it.x + (int64_t)rowid * it.ldx + un.a_lo, (uint32_t)(un.a_hi - un.a_lo) * 2u);
+                    if (un.b_hi > un.b_lo)
+                        bulk_prefetch_l2(it.yb + (int64_t)rowid * it.ldyb + un.b_lo, (uint32_t)(un.b_hi - un.b_lo) * 2u);
+                }
             }
         }
         if (!waited) {
@@ -214,12 +225,14 @@ __device__ __forceinline__ void producer(const FusedParams &P, unsigned char *sm
             }
             if (ok && !*dead) {
                 if (k < ja) p_request(P, smem, un, k, entry, st, rowid, lane, 0);
-                else p_request(P, smem, pend, pend.na + k - ja, pend_entry, st, pend_rowid, lane, 0);
+                else p_request(P, smem, pend, pend.na + k - ja, pend_entry, st, pend_rowid, lane, 0,
+                               !real && k == ja + jb - 1);   // nothing follows the last unit's last expand chunk
                 if (lane == 0) *count = q + 1;
             }
             ++q;
             if (++st == S) { st = 0; ++ph; }
         }
+        if (!real && jb > 0) sent_final = true;
         have_pend = un.run;
         pend = un;
         pend_rowid = rowid;
@@ -230,14 +243,17 @@ __device__ __forceinline__ void producer(const FusedParams &P, unsigned char *sm
         g = gn; u = un_; item = itn;
     }
     if (!waited) griddep_wait();
-    // end of the stream: a job without data
-    if (q >= S && ok) {
-        ok = mbar_wait(&empty[st], (ph - 1u) & 1u);
-        if (!ok) *dead = 1;
-    }
-    if (ok && !*dead && lane == 0) {
-        *reinterpret_cast<int4 *>(smem + SM_JOB + 16 * st) = make_int4(J_END, 0, 0, 0);
-        mbar_arrive(reinterpret_cast<uint64_t *>(smem + SM_FULL) + st);
+    // A stream without any job (no unit for this cluster, or units without expand chunks at its
+    // end) is closed by a job without data; otherwise the last expand chunk carried the mark.
+    if (!sent_final) {
+        if (q >= S && ok) {
+            ok = mbar_wait(&empty[st], (ph - 1u) & 1u);
+            if (!ok) *dead = 1;
+        }
+        if (ok && !*dead && lane == 0) {
+            *reinterpret_cast<int4 *>(smem + SM_JOB + 16 * st) = make_int4(J_END, 0, 0, 0);
+            mbar_arrive(reinterpret_cast<uint64_t *>(smem + SM_FULL) + st);
+        }
     }
     if (!ok && lane == 0) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
 }
@@ -441,6 +457,7 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[st]);
+            if (job.x & J_FINAL) break;
         }
         if (++st == P.n_stages) {
             st = 0;
@@ -521,8 +538,11 @@ decode_kernel(const __grid_constant__ FusedParams P) {
         fence_mbar_init();
     }
     __syncthreads();
-    // opening cluster barrier: arrived at here, waited for only where a block first touches a peer
-    cluster_arrive();
+    // Opening cluster barrier: arrived at here, waited for only where a block first touches a peer.
+    // Warp 0 (which set the barriers up) arrives with release; the others have nothing to publish
+    // and must not wait for their loads in flight.
+    if (warp == 0) cluster_arrive();
+    else cluster_arrive_relaxed();
     // Activations are only touched after griddep_wait().  The unit records and the pool were
     // complete before the preceding kernel started when P.early is set (the host sets it only
     // then), so they are read, and the first weight tiles requested, ahead of the wait.

@@ -480,7 +480,9 @@ lora_status_t launch_build_segments(lora_pool_t *pool, const int32_t *slot_idx_d
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
-    cfg.numAttrs = pool->tuning[2] == 1 ? 1 : 0;   // tuning key 2 = 1: programmatic dependent launch
+    // Programmatic dependent launch: the blocks may become resident while the kernel before them on
+    // the stream drains (they read nothing before griddepcontrol.wait); tuning key 2 = 2: never.
+    cfg.numAttrs = pool->tuning[2] != 2 ? 1 : 0;
     LORA_CUDA_TRY(cudaLaunchKernelEx(&cfg, build_segments_kernel, pool->view(), slot_idx_dev, T,
                                      tile_m, long_min, (int32_t *)meta_dev, staged));
     return count_launch();
