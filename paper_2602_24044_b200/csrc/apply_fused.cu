@@ -948,7 +948,10 @@ static lora_status_t launch_h(lora_pool_t *pool, FusedParams &P, int32_t C, cons
     P.n_stages = S;
     const int32_t smem = H == 0 ? dec::smem_bytes(S) : o;
     P.prefetch = pool->tuning[8] == 1 ? 0 : 1;
-    P.late_trigger = pool->tuning[11] == 1 ? 1 : 0;
+    // A launch of many projections runs for several waves of units; letting its successor's blocks
+    // in early only takes resources from its own later units (measured: -10 % on a seven-projection
+    // launch), while a short launch gains from the overlap.  Tuning key 11: 1 = never early, 2 = always.
+    P.late_trigger = pool->tuning[11] == 1 ? 1 : pool->tuning[11] == 2 ? 0 : P.n_items >= 4 ? 1 : 0;
     P.copy_idle = 0;
     for (int32_t i = 0; i < P.n_items; ++i) P.copy_idle |= P.item[i].in_place ? 0 : 1;
 
