@@ -61,6 +61,10 @@ def parse_args():
                     help="config 4: projections per launch: off = one lora_bgmv_apply each; groups = "
                          "{q,k,v} {o} {gate,up} {down} (the projections whose inputs exist together in a "
                          "transformer layer); layer = all seven of a layer in one lora_bgmv_apply_multi")
+    ap.add_argument("--sweep", action="store_true",
+                    help="instead of the benchmark line: apply latency against the number of distinct adapters, "
+                         "the rank and the batch size, and swap-in latency against the adapter size, with the "
+                         "linear fits the paper's performance model uses (Section 5.2, Eq. 1)")
     ap.add_argument("--layers", type=int, default=32,
                     help="config 4: transformer layers in the step (fewer only for profiling captures)")
     ap.add_argument("--tune", nargs="*", default=[], metavar="KEY=VALUE",
@@ -256,10 +260,158 @@ def case_workload(cfg, layers=32):
     return wl, rotation, n_proj
 
 
+# ---------------------------------------------------------------------------------------------
+# Sweep: the two estimators of the paper's performance model that this library's kernels
+# determine (Section 5.2, Eq. 1): the adapter overhead of the forward pass, modelled as linear in
+# the number of adapters in the batch (Overhead_A = K6 * A + K7, Section 5.1: linear growth, a jump
+# from no adapter to one, little influence of the rank), and Lat_load(S_A), the time to bring an
+# adapter of a given size from CPU memory.
+# ---------------------------------------------------------------------------------------------
+def run_sweep(args):
+    import torch
+    from paper_2602_24044_b200 import binding as lb
+    from paper_2602_24044_b200 import build as lbuild
+    from paper_2602_24044_b200 import workloads as W
+    from paper_2602_24044_b200.harness import Session, bf16_tensor
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(0)
+    lbuild.build()
+    dev = torch.device("cuda", 0)
+    sampler = ClockSampler(0)
+    sampler.start()
+    N, ROT, ACTS, D_IN, D_OUT, T_MAX = 128, 8, 32, 4096, 4096, 1024
+    out = {"sweep": "apply latency (one projection 4096->4096, cold: %d rotating weight copies, %d rotating "
+                    "activation sets) and swap-in latency" % (ROT, ACTS), "apply": [], "fits": [], "load": []}
+    rng = np.random.default_rng(26022404)
+    acts = [(torch.randn((T_MAX, D_IN), device=dev).to(torch.bfloat16),
+             torch.randn((T_MAX, D_OUT), device=dev).to(torch.bfloat16),
+             torch.empty((T_MAX, D_OUT), dtype=torch.bfloat16, device=dev)) for _ in range(ACTS)]
+
+    def time_graph(s, fn, n_calls):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s.compute):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(s.compute):
+            for _ in range(3):
+                g.replay()
+            a.record(s.compute)
+            g.replay()
+            b.record(s.compute)
+        torch.cuda.synchronize()
+        n = max(3, int(np.ceil(60.0 / max(a.elapsed_time(b), 1e-3))))
+        with torch.cuda.stream(s.compute):
+            a.record(s.compute)
+            for _ in range(n):
+                g.replay()
+            b.record(s.compute)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3 / (n * n_calls)
+
+    for rank in (8, 16, 32, 64):
+        wl = W.make_custom(T_MAX, D_IN, D_OUT, N, rank, r_max=64, scale=2.0, tile_m=8, seed=100 + rank)
+        wl.targets = wl.targets * ROT
+        wl.calls = list(range(ROT))
+        s = Session(wl, a_layout=lb.A_RANK_MAJOR, T_cap=T_MAX)
+        points = [(256, D) for D in (0, 1, 2, 4, 8, 16, 32, 64, 128)] + \
+                 [(T, min(T, 64)) for T in (64, 128, 512, 1024)]
+        for T, D in points:
+            # one table per slot group, so that consecutive applies use different adapters
+            groups = max(1, N // max(D, 1))
+            metas, sidx = [], []
+            for gidx in range(min(groups, 8)):
+                if D == 0:
+                    idx = np.full(T, -1, np.int32)
+                else:
+                    idx = (gidx * D + (np.arange(T) % D)).astype(np.int32)
+                    rng.shuffle(idx)
+                d = torch.from_numpy(idx).to(dev)
+                m = torch.empty(lb.segments_bytes(T, N, 8) // 4, dtype=torch.int32, device=dev)
+                lb.build_segments(s.pool, d, T, 8, 128, m, stream=s.compute)
+                metas.append(m)
+                sidx.append(d)
+            n_calls = ACTS
+
+            def calls():
+                for k in range(n_calls):
+                    x, yb, y = acts[k % ACTS]
+                    j = k % len(metas)
+                    lb.bgmv_apply(s.pool, k % ROT, x[:T], D_IN, yb[:T], D_OUT, y[:T], D_OUT, sidx[j], T,
+                                  metas[j], s.ws, stream=s.compute)
+            with torch.cuda.stream(s.compute):
+                calls()
+            torch.cuda.synchronize()
+            us = time_graph(s, calls, n_calls)
+            bytes_ = 2 * T * D_IN + (4 if D else 0) * T * D_OUT + 2 * D * rank * (D_IN + D_OUT)
+            out["apply"].append({"rank": rank, "T": T, "distinct_adapters": D, "us_per_apply": round(us, 3),
+                                 "algorithmic_MB": round(bytes_ / 1e6, 3),
+                                 "us_at_measured_peak": round(bytes_ / measured_peak()[0] * 1e-3, 3)})
+        st = lb.pool_check_status(s.pool, s.compute)
+        assert st[1] == 0, "a bounded device-side wait expired"
+        s.close()
+        pts = [(p["distinct_adapters"], p["us_per_apply"]) for p in out["apply"]
+               if p["rank"] == rank and p["T"] == 256 and p["distinct_adapters"] >= 1]
+        A = np.array([[d, 1.0] for d, _ in pts])
+        yv = np.array([u for _, u in pts])
+        (k6, k7), res, _, _ = np.linalg.lstsq(A, yv, rcond=None)
+        zero = [p["us_per_apply"] for p in out["apply"] if p["rank"] == rank and p["T"] == 256
+                and p["distinct_adapters"] == 0][0]
+        pred = A @ np.array([k6, k7])
+        out["fits"].append({"rank": rank, "T": 256, "model": "us = K6 * A + K7 over A = 1 .. 128 adapters in the batch",
+                            "K6_us_per_adapter": round(float(k6), 4), "K7_us": round(float(k7), 3),
+                            "max_abs_residual_us": round(float(np.abs(pred - yv).max()), 3),
+                            "us_without_adapter": round(zero, 3),
+                            "jump_0_to_1_us": round(pts[0][1] - zero, 3),
+                            "bytes_model_slope_us_per_adapter": round(2 * rank * (D_IN + D_OUT) / measured_peak()[0] * 1e-3, 4)})
+
+    # Lat_load: one adapter of Llama-3-8B shape (7 projections x 32 layers) from pinned host memory
+    targets = W.LLAMA3_8B_TARGETS * 32
+    for rank in (8, 16, 32, 64):
+        wl = W.make_custom(8, 64, 64, 2, rank, r_max=rank, seed=200 + rank)
+        wl.targets = targets
+        wl.calls = [0]
+        wl.weight_mode = "lora"
+        s = Session(wl, slots=[])
+        per = sum(a + b for a, b in targets) * rank * 2
+        packed = torch.empty(per // 2, dtype=torch.bfloat16).pin_memory()
+        mats_a = [torch.empty((rank, a), dtype=torch.bfloat16).pin_memory() for a, _ in targets]
+        mats_b = [torch.empty((rank, b), dtype=torch.bfloat16).pin_memory() for _, b in targets]
+        res = {}
+        for name, A_, B_, layout in (("one_buffer", [packed] * len(targets), [packed] * len(targets), lb.PACKED),
+                                     ("per_matrix", mats_a, mats_b, lb.A_RANK_MAJOR)):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            lb.pool_load_slot(s.pool, 0, rank, 2.0, A_, B_, layout, s.load, None, True)
+            torch.cuda.synchronize()
+            reps = 3
+            a.record(s.load)
+            for k in range(reps):
+                lb.pool_load_slot(s.pool, k % 2, rank, 2.0, A_, B_, layout, s.load, None, True)
+            b.record(s.load)
+            torch.cuda.synchronize()
+            res[name] = a.elapsed_time(b) / reps
+        out["load"].append({"rank": rank, "adapter_MB": round(per / 1e6, 1),
+                            "ms_one_buffer": round(res["one_buffer"], 3), "ms_per_matrix": round(res["per_matrix"], 3),
+                            "GBps_one_buffer": round(per / res["one_buffer"] / 1e6, 1),
+                            "GBps_per_matrix": round(per / res["per_matrix"] / 1e6, 1)})
+        s.close()
+    ld = out["load"]
+    A = np.array([[p["adapter_MB"], 1.0] for p in ld])
+    (m, c), _, _, _ = np.linalg.lstsq(A, np.array([p["ms_one_buffer"] for p in ld]), rcond=None)
+    out["fits"].append({"model": "Lat_load ms = a * S_A[MB] + b (one pinned buffer per adapter)",
+                        "a_ms_per_MB": round(float(m), 5), "b_ms": round(float(c), 3)})
+    out["clocks"] = sampler.stop()
+    out["peak_GBps"] = measured_peak()[0]
+    print(json.dumps(out))
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.sweep:
+        return run_sweep(args)
 
     import torch
     import torch.distributed as dist

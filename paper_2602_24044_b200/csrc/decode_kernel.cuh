@@ -483,12 +483,27 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
             if (!meet()) break;
             if (tid < rows) rowidx[tid] = __ldg(P.meta + P.moff_perm + (P.T - n_idle) + first + tid);
             if (!meet()) break;
+            // the chunk's rows as one index space (row, 16-byte vector of this block's share), four
+            // independent loads in flight per thread
             const int32_t vecs = it.d_out / 8;
-            for (int32_t m = 0; m < rows; ++m) {
-                const __nv_bfloat16 *src = it.yb + (int64_t)rowidx[m] * it.ldyb;
-                __nv_bfloat16 *dst = it.y + (int64_t)rowidx[m] * it.ldy;
-                for (int32_t v = (int32_t)crank * FT + tid; v < vecs; v += (int32_t)csize * FT)
-                    reinterpret_cast<uint4 *>(dst)[v] = ldg16(src + (int64_t)v * 8);
+            const int32_t per_blk = (vecs + (int32_t)csize - 1) / (int32_t)csize;
+            const int32_t v_lo = (int32_t)crank * per_blk, v_n = max(0, min(per_blk, vecs - v_lo));
+            const int32_t total = rows * v_n;
+            for (int32_t i0 = tid; i0 < total; i0 += 4 * FT) {
+                uint4 val[4];
+                int64_t off[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int32_t i = i0 + q * FT;
+                    const int32_t m = i < total ? i / v_n : 0, v = i < total ? v_lo + i - m * v_n : 0;
+                    off[q] = (int64_t)rowidx[m];
+                    val[q] = make_uint4(0, 0, 0, 0);
+                    if (i < total) val[q] = ldg16(it.yb + off[q] * it.ldyb + (int64_t)v * 8);
+                    off[q] = off[q] * it.ldy + (int64_t)v * 8;
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (i0 + q * FT < total) *reinterpret_cast<uint4 *>(it.y + off[q]) = val[q];
             }
         }
     }
