@@ -120,7 +120,10 @@ typedef struct {
  * rows 0 .. rank-1 meaningful, the rest zero.  LORA_A_DIN_MAJOR input is transposed on the device.
  * Host matrices must stay valid until the ready event has fired (lora_pool_acquire + stream
  * completion, or a synchronise on load_stream).  compute_stream may be NULL when no reader
- * can be in flight.  On any error the slot is left untouched.
+ * can be in flight.  All loads of one pool go through ONE load stream (LORA_A_DIN_MAJOR input
+ * passes through a staging area of the pool that consecutive loads reuse in stream order).
+ * On an argument error (every code below but CUDA) the slot is left untouched; after a CUDA error
+ * in the middle of the sequence the slot is empty on the device and in the host's view.
  * Errors: INVALID_ARG, SLOT_RANGE, RANK, NOT_PINNED, CUDA.
  */
 lora_status_t lora_pool_load_slot(lora_pool_t *pool, int32_t slot, const lora_adapter_host_t *adapter,
@@ -176,6 +179,9 @@ lora_status_t lora_pool_selftest_wait_expiry(lora_pool_t *pool, int32_t polls, i
  *   key 7  segment builder: 1 = one warp per slot also for long batches
  *   key 8  fused kernel: 1 = no L2 hints ahead of the shared-memory ring
  *   key 9  fused kernel: share (1 .. 99 %) of the resident clusters one launch may take
+ *   key 10 1 = decode batches take the general fused kernel, not the decode kernel
+ *   key 11 when a fused kernel lets its successor on the stream become resident: 1 = only at its
+ *          end, 2 = at its start (default: at its start for launches of fewer than four projections)
  * Keys outside 0 .. 15 -> INVALID_ARG. */
 lora_status_t lora_pool_set_tuning(lora_pool_t *pool, int32_t key, int32_t value);
 
@@ -248,8 +254,8 @@ lora_status_t lora_pool_plan(size_t bytes_budget, const lora_target_t *targets, 
  *                flags bit0: the segment's tokens are consecutive ids; bit1: length >= long_min
  *   tile_seg[cap_tile], tile_row0[cap_tile], tile_rows[cap_tile]
  *                each segment cut into pieces of at most tile_m rows (positions in perm)
- *   tile_flags[cap_tile]   bit0: the tile's tokens are consecutive ids
- *   (then, from the next 16-byte boundary, words private to the library: a 4-word record per
+ *   (then words private to the library: one flag word per tile, and from the next 16-byte
+ *    boundary a 4-word record per
  *    tile, and a 4-word record plus 16 row ids per piece of at most 16 rows of a tile;
  *    lora_segments_bytes counts them)
  * Unused entries are -1.  A token is active iff its slot id names an occupied slot; a token

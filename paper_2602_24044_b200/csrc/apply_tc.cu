@@ -528,18 +528,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapFloatOOBfill);
 
 static EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
+    // looked up once per process; a function-local static is initialised under the language's own lock
+    static const EncodeTiledFn fn = [] {
         void *p = nullptr;
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
             q == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
-        else
-            cudaGetLastError();
-    }
+            return (EncodeTiledFn)p;
+        cudaGetLastError();
+        return (EncodeTiledFn) nullptr;
+    }();
     return fn;
 }
 
@@ -581,8 +579,7 @@ static lora_status_t launch_tc_bucket(lora_pool_t *pool, const TcParams &P, cons
         return LORA_ERR_INVALID_ARG;
 
     constexpr int SH_SMEM = SH_STAGES * (XT_BYTES + ((RP * 128 + 1023) & ~1023)) + 256 + 1024;
-    static bool attr_done_d[DEVICE_TABLE] = {};
-    bool &attr_done = attr_done_d[device_index(pool->device)];
+    bool &attr_done = pool->tc_attr_done[RP == 16 ? 0 : RP == 32 ? 1 : 2];
     if (!attr_done) {
         LORA_CUDA_TRY(cudaFuncSetAttribute(tc_shrink_kernel<RP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            SH_SMEM));

@@ -219,8 +219,7 @@ lora_status_t launch_twophase(lora_pool_t *pool, ApplyParams &P, void *workspace
     P.JS = JS;
     P.ws = (float *)workspace;
 
-    static bool attr_done_d[DEVICE_TABLE] = {};
-    bool &attr_done = attr_done_d[device_index(pool->device)];
+    bool &attr_done = pool->twophase_attr_done;
     if (!attr_done) {
         LORA_CUDA_TRY(cudaFuncSetAttribute(shrink_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            TP_SMEM_BYTES));

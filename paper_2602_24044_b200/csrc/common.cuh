@@ -148,6 +148,10 @@ struct lora_pool {
         int32_t attr_smem = 0, occ_smem = 0, occ_c = 0, occ_clusters = 0;
     };
     FusedLaunchCache fused_cache[3];
+    // kernel attributes the other launchers have set for this pool's device
+    bool twophase_attr_done = false;
+    bool tc_attr_done[3] = {false, false, false};   // rank buckets 16, 32, 64
+    size_t seg_attr_smem = 0, seg_attr_chunked = 0;
 
     // Shapes of the metadata tables built through this handle (the table itself lives on the
     // device; apply calls need T and tile_m on the host to size their grids).

@@ -229,6 +229,9 @@ lora_status_t lora_pool_load_slot(lora_pool_t *pool, int32_t slot, const lora_ad
 
     set_slot_kernel<<<1, 32, 0, ls>>>(pool->table_dev, slot, 0, 0.0f, 0);
     if ((s = count_launch()) != LORA_OK) return s;
+    // from here on the slot is empty on the device; the host's view follows until the load is
+    // queued completely (an error on the way leaves both sides saying "empty")
+    pool->table_host[slot] = {0, 0.0f, 0, 0};
 
     // One DMA per matrix.  Neighbouring host matrices given as separate pointers are not merged
     // into one copy: two pinned allocations can be adjacent in the address space, and a copy must

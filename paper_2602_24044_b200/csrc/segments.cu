@@ -439,8 +439,7 @@ lora_status_t launch_build_segments(lora_pool_t *pool, const int32_t *slot_idx_d
         const size_t words = 6 * (size_t)N + (size_t)T + (size_t)C * (N + 1) + 2 * (size_t)L.cap_tile;
         if (words * sizeof(int32_t) <= 200 * 1024) {
             const size_t smem = words * sizeof(int32_t);
-            static size_t attr_chunked_d[DEVICE_TABLE] = {};
-            size_t &attr_chunked = attr_chunked_d[device_index(pool->device)];
+            size_t &attr_chunked = pool->seg_attr_chunked;
             if (attr_chunked == 0) attr_chunked = 48 * 1024;
             if (smem > attr_chunked) {
                 cudaError_t e = cudaFuncSetAttribute(build_segments_chunked_kernel,
@@ -462,8 +461,7 @@ lora_status_t launch_build_segments(lora_pool_t *pool, const int32_t *slot_idx_d
     // the token list is copied to shared memory when it fits beside the per-slot arrays
     const int32_t staged = sizeof(int32_t) * (6 * (size_t)N + (size_t)T) <= 200 * 1024 ? 1 : 0;
     const size_t smem = sizeof(int32_t) * (6 * (size_t)N + (staged ? (size_t)T : 0));
-    static size_t attr_smem_d[DEVICE_TABLE] = {};
-    size_t &attr_smem = attr_smem_d[device_index(pool->device)];
+    size_t &attr_smem = pool->seg_attr_smem;
     if (attr_smem == 0) attr_smem = 48 * 1024;
     if (smem > attr_smem) {
         cudaError_t e = cudaFuncSetAttribute(build_segments_kernel,
