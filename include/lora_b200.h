@@ -175,9 +175,9 @@ lora_status_t lora_pool_selftest_wait_expiry(lora_pool_t *pool, int32_t polls, i
  *   key 3  fused kernel: upper bound on the clusters in the grid
  *   key 4  tensor-core kernels of lora_sgmv_apply: 1 = never, 2 = whenever they apply
  *   key 5  fused kernel: stages of the shared-memory ring (2 .. 4)
- *   key 6  fused kernel: 1 = partial sums always fetched from the cluster's blocks, never pushed
+ *   key 6  (unused)
  *   key 7  segment builder: 1 = one warp per slot also for long batches
- *   key 8  fused kernel: 1 = no L2 hints ahead of the shared-memory ring
+ *   key 8  (unused)
  *   key 9  fused kernel: share (1 .. 99 %) of the resident clusters one launch may take
  *   key 10 1 = decode batches take the general fused kernel, not the decode kernel
  *   key 11 when a fused kernel lets its successor on the stream become resident: 1 = only at its

@@ -301,7 +301,7 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
     auto meet = [&]() {
         uint64_t *cb = reinterpret_cast<uint64_t *>(smem + SM_CBAR);
         mbar_arrive(cb);
-        const bool done = mbar_wait(cb, cs & 1u);
+        const bool done = __all_sync(0xffffffffu, mbar_wait(cb, cs & 1u));
         ++cs;
         if (!done) *dead = 1;
         return done && !*dead;
@@ -309,7 +309,7 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
     if (P.early) griddep_wait();
 
     for (;;) {
-        ok = mbar_wait(&full[st], ph & 1u);
+        ok = __all_sync(0xffffffffu, mbar_wait(&full[st], ph & 1u));   // a warp stays together
         if (!ok) {
             *dead = 1;
             break;
@@ -343,7 +343,8 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
                 // ---- the block's partial goes to every block of the cluster (buffer set kp & 1) ----
                 const int b = kp & 1;
                 if (kp >= 2) {   // the peers have read what this set held two units ago
-                    ok = mbar_wait_cluster(reinterpret_cast<uint64_t *>(smem + SM_YB) + b, (uint32_t)((kp - 2) >> 1) & 1u);
+                    ok = __all_sync(0xffffffffu, mbar_wait_cluster(reinterpret_cast<uint64_t *>(smem + SM_YB) + b,
+                                                                   (uint32_t)((kp - 2) >> 1) & 1u));
                     if (!ok) {
                         *dead = 1;
                         break;
@@ -373,7 +374,8 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
             if (job.x & J_FIRST) {
                 // ---- every block sums the cluster's partials in block order (buffer set kr & 1) ----
                 const int b = kr & 1;
-                ok = mbar_wait_cluster(reinterpret_cast<uint64_t *>(smem + SM_XB) + b, (uint32_t)(kr >> 1) & 1u);
+                ok = __all_sync(0xffffffffu, mbar_wait_cluster(reinterpret_cast<uint64_t *>(smem + SM_XB) + b,
+                                                               (uint32_t)(kr >> 1) & 1u));
                 if (!ok) {
                     *dead = 1;
                     break;
