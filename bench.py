@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None: no capture of the current kernel on that workload)
-NCU_TRAFFIC = {1: 22.9e6}
+NCU_TRAFFIC = {1: 22.9e6, (4, "layer"): 269.4e6, 3: 175.3e6}
 
 PAPER_CONTEXT = {
     "note": "system-level results of the paper, other hardware, context only",
@@ -727,10 +727,12 @@ def main():
             "frac": achieved / peak, "peak_source": "%s copy bandwidth" % peak_kind,
             "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
             "kernel": ("shrink_kernel + expand_kernel (two launches per apply)" if not fused
-                       else "tc_shrink_kernel + tc_expand_kernel + fused_kernel (one apply; tc_expand dominates)"
-                       if cfg == 2 else "fused_kernel (one launch per apply, every rank)"),
+                       else "tc_shrink_kernel + tc_expand_kernel + stream_kernel (one apply; tc_expand dominates)"
+                       if cfg == 2 else "stream_kernel (one launch per apply, every rank)" if cfg == 3
+                       else "decode_kernel (one launch per %s)" % ("apply" if launches_multi is None else
+                                                                    "layer" if multi == "layer" else "group of projections")),
             "algorithmic_bytes_per_launch": alg / launches_per_step,
-            "us_per_launch": apply_ms * 1e3, "traffic": NCU_TRAFFIC.get(cfg) if fused else None,
+            "us_per_launch": apply_ms * 1e3, "traffic": NCU_TRAFFIC.get((4, multi) if cfg == 4 else cfg) if fused else None,
             "averaged_over": "%d launches per step" % launches_per_step,
             "warm_l2_us_per_launch": warm_us,
         },
