@@ -24,12 +24,14 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
     int32_t *tile0 = segid + N;    // [N] first tile number
     int32_t *occ = tile0 + N;      // [N] slot occupied (copy of the slot table's flag)
     int32_t *piece0 = occ + N;     // [N] first 16-row piece number
-    int32_t *tok = piece0 + N;     // [T] copy of the token list (only when `staged`)
+    const MetaLayout L = meta_layout(T, N, tile_m);
+    int32_t *tfirst = piece0 + N;          // [cap_tile] first token id of a tile
+    int32_t *tlast = tfirst + L.cap_tile;  // [cap_tile] last token id of a tile
+    int32_t *tok = tlast + L.cap_tile;     // [T] copy of the token list (only when `staged`)
     __shared__ int32_t warp_tot[4][SEG_WARPS];
     __shared__ int32_t totals[4];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const MetaLayout L = meta_layout(T, N, tile_m);
     // programmatic dependent launch: the next kernel of the stream may be scheduled now; this one
     // waits until everything queued before it is complete (no-ops without the launch attribute)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -110,6 +112,9 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
         const int32_t n = cnt[s];
         if (n == 0) continue;
         const int32_t p0 = start[s], seg = segid[s];
+        // the slot's rank and scale for the records below: asked for now, needed after the scan, so
+        // that this trip to global memory is off the critical path
+        const int4 slot_entry = __ldg(reinterpret_cast<const int4 *>(pool.table + s));
         int32_t run = 0;
         // 128 tokens per step: the four loads are independent, the ballots keep token order
         for (int32_t base = 0; base < T && run < n; base += 128) {
@@ -130,19 +135,23 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
                     // private copy laid out by unit (16-row piece of a tile), 16 ids per unit
                     const int32_t k = j / tile_m, jj = j - k * tile_m;
                     meta[L.unit_perm + 16 * (int64_t)(piece0[s] + k * ppt + (jj >> 4)) + (jj & 15)] = t;
+                    // first and last token of every tile, kept on chip: what was just stored to
+                    // global memory is not read back
+                    if (jj == 0) tfirst[tile0[s] + k] = t;
+                    if (jj == tile_m - 1 || j == n - 1) tlast[tile0[s] + k] = t;
                 }
                 run += __popc(m);
             }
         }
         __syncwarp();
-        const int32_t first = perm[p0], last = perm[p0 + n - 1];
+        const int32_t nt = (n + tile_m - 1) / tile_m;
+        const int32_t first = tfirst[tile0[s]], last = tlast[tile0[s] + nt - 1];
         if (lane == 0) {
             meta[L.seg_slot + seg] = s;
             meta[L.seg_start + seg] = p0;
-            meta[L.seg_rank + seg] = pool.table[s].rank;
+            meta[L.seg_rank + seg] = slot_entry.x;
             meta[L.seg_flags + seg] = (last - first + 1 == n ? 1 : 0) | (n >= long_min ? 2 : 0);
         }
-        const int32_t nt = (n + tile_m - 1) / tile_m;
         for (int32_t k = lane; k < nt; k += 32) {
             const int32_t r0 = p0 + k * tile_m;
             const int32_t rows = min(tile_m, p0 + n - r0);
@@ -150,9 +159,11 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
             meta[L.tile_seg + idx] = seg;
             meta[L.tile_row0 + idx] = r0;
             meta[L.tile_rows + idx] = rows;
-            const int32_t contiguous = (perm[r0 + rows - 1] - perm[r0] + 1 == rows) ? 1 : 0;
+            const int32_t contiguous = (tlast[idx] - tfirst[idx] + 1 == rows) ? 1 : 0;
             meta[L.tile_flags + idx] = contiguous;
-            const SlotEntry e = pool.table[s];
+            SlotEntry e;
+            e.rank = slot_entry.x;
+            e.scale = __int_as_float(slot_entry.y);
             // private record: slot, position, rows (bits 0-14) | consecutive ids (bit 15) | rank, scale
             *reinterpret_cast<int4 *>(meta + L.tile_desc + 4 * (int64_t)idx) =
                 make_int4(s, r0, rows | (contiguous << 15) | (e.rank << 16), __float_as_int(e.scale));
@@ -459,8 +470,9 @@ lora_status_t launch_build_segments(lora_pool_t *pool, const int32_t *slot_idx_d
     if (grid > 2 * pool->sm_count) grid = 2 * pool->sm_count;
     if (grid < 1) grid = 1;
     // the token list is copied to shared memory when it fits beside the per-slot arrays
-    const int32_t staged = sizeof(int32_t) * (6 * (size_t)N + (size_t)T) <= 200 * 1024 ? 1 : 0;
-    const size_t smem = sizeof(int32_t) * (6 * (size_t)N + (staged ? (size_t)T : 0));
+    const size_t fixed = 6 * (size_t)N + 2 * (size_t)meta_layout(T, N, tile_m).cap_tile;
+    const int32_t staged = sizeof(int32_t) * (fixed + (size_t)T) <= 200 * 1024 ? 1 : 0;
+    const size_t smem = sizeof(int32_t) * (fixed + (staged ? (size_t)T : 0));
     size_t &attr_smem = pool->seg_attr_smem;
     if (attr_smem == 0) attr_smem = 48 * 1024;
     if (smem > attr_smem) {
