@@ -243,16 +243,21 @@ tc_shrink_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_x,
     const uint32_t tmem = *tmem_slot;
     bool ok = true;
 
-    if (tid == 0 && nkb > 0) {
-        constexpr uint32_t IDESC = tc::instr_desc(128, RP, 0, 0);
-        auto issue_load = [&](int32_t i) {
+    // Two single-thread roles in different warps: one requests tiles (it alone waits for a stage
+    // to be read out before refilling it), one issues the MMAs (it only ever waits for data).
+    if (tid == 32 && nkb > 0) {
+        for (int32_t i = 0; i < nkb && ok; ++i) {
             const int s = i % SH_STAGES;
+            if (i >= SH_STAGES) ok = tc::mbar_wait(&empty[s], (uint32_t)(i / SH_STAGES - 1) & 1u);
+            if (!ok) break;
             unsigned char *st = smem + s * STAGE;
             tc::mbar_expect_tx(&full[s], XT_BYTES + AT_BYTES);
             tc::tma_load_2d(st, &map_x, (kb0 + i) * 64, lt.t0, &full[s]);
             tc::tma_load_3d(st + XT_BYTES, &map_a, (kb0 + i) * 64, 0, lt.slot, &full[s]);
-        };
-        for (int32_t i = 0; i < nkb && i < SH_STAGES; ++i) issue_load(i);
+        }
+    }
+    if (tid == 0 && nkb > 0) {
+        constexpr uint32_t IDESC = tc::instr_desc(128, RP, 0, 0);
         for (int32_t i = 0; i < nkb && ok; ++i) {
             const int s = i % SH_STAGES;
             const uint32_t ph = (uint32_t)(i / SH_STAGES) & 1u;
@@ -266,11 +271,7 @@ tc_shrink_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_x,
                 const uint64_t bd = tc::smem_desc(aa + k4 * 32, 16, 1024, tc::LAYOUT_SW128);
                 tc::umma(tmem, ad, bd, IDESC, (i > 0 || k4 > 0) ? 1u : 0u);
             }
-            tc::umma_commit(&empty[s]);
-            if (i + SH_STAGES < nkb) {       // refill this stage once the MMAs have read it
-                ok = tc::mbar_wait(&empty[s], ph);
-                if (ok) issue_load(i + SH_STAGES);
-            }
+            tc::umma_commit(&empty[s]);   // the stage may be refilled once these MMAs have read it
         }
         tc::umma_commit(done);
     }
