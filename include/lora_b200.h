@@ -277,8 +277,9 @@ lora_status_t lora_build_segments(lora_pool_t *pool, const int32_t *slot_idx_dev
  * not overlapping it.  Tokens without an active slot get y = y_base bit for bit.  Row t of y
  * depends only on row t of x and y_base, the token's slot and the pool.
  * workspace: dev scratch of >= lora_workspace_bytes(pool, T) bytes (fp32 partial products
- * v = x . A_i between the two phases of the tensor-core and two-phase kernels; the fused kernel
- * keeps v on chip), contents undefined afterwards; calls sharing a workspace must be ordered on
+ * v = x . A_i between the two phases of the tensor-core and two-phase kernels and the
+ * tensor-core path's list of long tiles; the fused kernels keep v on chip), contents undefined
+ * afterwards; calls sharing a workspace must be ordered on
  * one stream.
  * Ordering: every apply is ordered behind the lora_build_segments call that wrote its table.
  * Later applies on the same table may start reading the table and the pool (never x or y_base)

@@ -172,20 +172,27 @@ struct TcParams {
     int32_t target_rows;    // r_max: rows of a slot's matrices
     __nv_bfloat16 *y;       // output, for tiles with fewer than 128 rows (stored row by row)
     int64_t ldy;
+    int32_t *list;          // work list in the workspace: [0] = number of long tiles, then their tile numbers
+    int32_t list_cap;
 };
 
 // tile record -> (valid long tile of this bucket?, slot, first token, position in perm, rank, scale)
 constexpr int TC_MIN_ROWS = 32;    // shortest run of consecutive tokens given to the tensor cores
+// Batches of fewer than this many 128-row tiles do not come here: a handful of long tiles cannot
+// fill the GPU with 128-row blocks, and the three extra launches cost more than they save
+// (mixed chunked-prefill batch with sixteen long tiles: 127 us with them, 97 us on the stream kernel alone).
+constexpr int TC_MIN_TILES = 32;
 struct LongTile {
     int32_t slot, t0, row0, rank, rows;
     float scale;
     bool ok;
 };
-__device__ __forceinline__ LongTile long_tile(const TcParams &P, int32_t unit) {
+// entry: position in the work list (the grid is sized by a bound on the list's length)
+__device__ __forceinline__ LongTile long_tile(const TcParams &P, int32_t entry) {
     LongTile lt;
     lt.ok = false;
-    const int32_t n_tile = __ldg(P.meta + H_NTILE);
-    if (unit >= n_tile) return lt;
+    if (entry >= P.list[0]) return lt;
+    const int32_t unit = P.list[1 + entry];
     const int4 d = __ldg(reinterpret_cast<const int4 *>(P.meta + P.moff_desc) + unit);
     const int32_t rows = d.z & 0x7fff, contiguous = (d.z >> 15) & 1, rank = d.z >> 16;
     if (d.x < 0 || rows < TC_MIN_ROWS || !contiguous) return lt;
@@ -197,6 +204,42 @@ __device__ __forceinline__ LongTile long_tile(const TcParams &P, int32_t unit) {
     lt.t0 = __ldg(P.meta + P.moff_perm + d.y);
     lt.ok = true;
     return lt;
+}
+
+// The tiles this path takes (runs of at least TC_MIN_ROWS consecutive tokens), in tile order, as a
+// compact list: the two kernels below then launch one block column per list entry instead of one
+// per tile of the batch (a mixed batch has hundreds of tiles and a handful of long ones).
+__global__ void __launch_bounds__(256)
+tc_worklist_kernel(const TcParams P) {
+    __shared__ int32_t warp_count[8];
+    __shared__ int32_t base_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t n_tile = P.meta[H_NTILE];
+    if (tid == 0) base_s = 0;
+    __syncthreads();
+    for (int32_t t0 = 0; t0 < n_tile; t0 += 256) {
+        const int32_t idx = t0 + tid;
+        bool take = false;
+        if (idx < n_tile) {
+            const int4 d = *(reinterpret_cast<const int4 *>(P.meta + P.moff_desc) + idx);
+            take = d.x >= 0 && (d.z & 0x7fff) >= TC_MIN_ROWS && ((d.z >> 15) & 1);
+        }
+        const uint32_t m = __ballot_sync(0xffffffffu, take);
+        if (lane == 0) warp_count[warp] = __popc(m);
+        __syncthreads();
+        int32_t before = base_s;
+        for (int w = 0; w < warp; ++w) before += warp_count[w];
+        const int32_t pos = before + __popc(m & ((1u << lane) - 1u));
+        if (take && pos < P.list_cap) P.list[1 + pos] = idx;
+        __syncthreads();
+        if (tid == 0) {
+            int32_t tot = 0;
+            for (int w = 0; w < 8; ++w) tot += warp_count[w];
+            base_s += tot;
+        }
+        __syncthreads();
+    }
+    if (tid == 0) P.list[0] = min(base_s, P.list_cap);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -602,11 +645,9 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
                                    size_t workspace_bytes, cudaStream_t stream, bool *handled) {
     *handled = false;
     if (!AP.meta || AP.tile_m != TC_ROWS || AP.T < TC_ROWS) return LORA_OK;
-    // Fewer than ~32 full tiles cannot fill the GPU with 128-row blocks (the grids below are sized
-    // by a bound on the tile count, not the count itself); the fused kernel alone was measured
-    // faster there (mixed chunked-prefill batch: 108 us against 166 us).  Tuning key 4 = 2 forces
-    // this path whenever it applies.
-    if (AP.T / TC_ROWS < 32 && pool->tuning[4] != 2) return LORA_OK;
+    // Short batches stay on the stream kernel alone (tuning key 4 = 2 forces this path whenever it
+    // applies).
+    if (AP.T / TC_ROWS < TC_MIN_TILES && pool->tuning[4] != 2) return LORA_OK;
     if (!encode_fn()) return LORA_OK;
     // TMA wants 16-byte aligned bases and row pitches
     if ((((uintptr_t)AP.x | (uintptr_t)AP.yb | (uintptr_t)AP.y) & 15) || (AP.ldx % 8) || (AP.ldyb % 8) ||
@@ -621,8 +662,11 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
     const int32_t nkb = (AP.tv.d_in + 63) / 64;
     while (KS > 1 && KS > nkb) KS >>= 1;
     const size_t per_split = (size_t)AP.T * RS * sizeof(float);
-    while (KS > 1 && per_split * KS > workspace_bytes) KS >>= 1;
-    if (!workspace || per_split * KS > workspace_bytes || ((uintptr_t)workspace & 15)) return LORA_OK;
+    // the work list (count + tile numbers) sits at the end of the workspace
+    const size_t list_bytes = (((size_t)max_long + 1) * sizeof(int32_t) + 15) & ~(size_t)15;
+    if (!workspace || workspace_bytes < list_bytes + per_split || ((uintptr_t)workspace & 15)) return LORA_OK;
+    const size_t ws_partials = (workspace_bytes - list_bytes) & ~(size_t)15;
+    while (KS > 1 && per_split * KS > ws_partials) KS >>= 1;
     int32_t NS = (4 * pool->sm_count + max_long - 1) / max_long;
     const int32_t nblk = (AP.tv.d_out + 63) / 64;
     if (NS > nblk) NS = nblk;
@@ -642,7 +686,14 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
     P.moff_perm = (int32_t)L.perm;
     P.moff_desc = (int32_t)L.tile_desc;
     P.target_rows = pool->r_max;
-    const int32_t units = L.cap_tile;
+    P.list = reinterpret_cast<int32_t *>((char *)workspace + ws_partials);
+    P.list_cap = max_long;
+    const int32_t units = max_long;   // block columns: one per work-list entry, the unused ones leave at once
+    tc_worklist_kernel<<<1, 256, 0, stream>>>(P);
+    {
+        lora_status_t sl = count_launch();
+        if (sl != LORA_OK) return sl;
+    }
 
     P.y = AP.y;
     P.ldy = AP.ldy;
