@@ -288,8 +288,9 @@ tc_shrink_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_x,
 
     // Two single-thread roles in different warps: one requests tiles (it alone waits for a stage
     // to be read out before refilling it), one issues the MMAs (it only ever waits for data).
+    int32_t issued = 0;   // tiles requested by the loading thread
     if (tid == 32 && nkb > 0) {
-        for (int32_t i = 0; i < nkb && ok; ++i) {
+        for (int32_t i = 0; i < nkb && ok; ++i, ++issued) {
             const int s = i % SH_STAGES;
             if (i >= SH_STAGES) ok = tc::mbar_wait(&empty[s], (uint32_t)(i / SH_STAGES - 1) & 1u);
             if (!ok) break;
@@ -344,8 +345,13 @@ tc_shrink_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_x,
                     *reinterpret_cast<uint4 *>(dst + c + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
             }
         }
-    } else if (tid == 0) {
-        atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
+    } else {
+        if (tid == 0) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
+        // copies still on their way into this block's shared memory must land before it leaves:
+        // the most recent request of every stage is waited for (bounded)
+        if (tid == 32)
+            for (int32_t q = max(issued - SH_STAGES, 0); q < issued; ++q)
+                tc::mbar_wait(&full[q % SH_STAGES], (uint32_t)(q / SH_STAGES) & 1u);
     }
     tc::tc_fence_before();
     __syncthreads();
@@ -480,17 +486,27 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
         // ---- producer: one thread requests tiles S - 2 blocks ahead and issues each block's MMAs
         // as soon as its tiles have landed; it never waits for an epilogue that is under way ------
         if (lane == 0) {
-            for (int32_t j = 0; j < nblk && j < S - 2; ++j) issue_load(j);
+            int32_t issued = 0;
+            for (int32_t j = 0; j < nblk && j < S - 2; ++j, ++issued) issue_load(j);
             for (int32_t j = 0; j < nblk && ok; ++j) {
                 if (*failed) break;
                 ok = issue_mma(j);
                 const int32_t n = j + S - 2;          // next block to request
                 if (ok && n < nblk) {
                     if (n >= S) ok = tc::mbar_wait(&freed[n % S], (uint32_t)(n / S - 1) & 1u);
-                    if (ok) issue_load(n);
+                    if (ok) {
+                        issue_load(n);
+                        ++issued;
+                    }
                 }
             }
-            if (!ok) *failed = 1;
+            if (!ok || *failed) {
+                *failed = 1;
+                // copies still on their way into this block's shared memory must land before it
+                // leaves: the most recent request of every stage is waited for (bounded)
+                for (int32_t q = max(issued - S, 0); q < issued; ++q)
+                    tc::mbar_wait(&full[q % S], (uint32_t)(q / S) & 1u);
+            }
         }
         __syncwarp();
     } else {
