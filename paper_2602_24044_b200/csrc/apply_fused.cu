@@ -32,7 +32,8 @@ constexpr int FT = 128;          // consumer threads per block (four warps)
 constexpr int FT_ALL = 160;      // plus the warp that requests the jobs
 constexpr int SM_HEADER = 1024;  // general kernel: barriers, job headers and unit entries come before the carved-up buffers
 constexpr int MAX_STAGES = 4;
-constexpr int W_BYTES = 8192;    // weight tile of a job: rank bucket x chunk width x 2 bytes, for every bucket
+constexpr int W_BYTES = 8192;    // decode kernel: weight tile of a job, 16 rank rows x 256 columns x 2 bytes
+constexpr int GEN_W_BYTES = 16384;   // general kernel: 32 rank rows x 256 columns or 64 x 128
 constexpr int TOK_PITCH = 256 + 8;   // elements between token rows of a stage (+16 B against bank conflicts)
 constexpr int MAPS_PER_TARGET = 16;  // tensor maps of a target: A then B, index rows / 8 - 1 for loads of 8 .. 64 rank rows
 constexpr int MAX_ITEMS = 8;
@@ -65,6 +66,7 @@ struct FusedParams {
     int32_t copy_idle;         // some projection is out of place: rows without adapter are copied
     int32_t off_part, off_vpart, vbuf_bytes, off_vh, off_vl;   // warp partials, exchange buffers (x2), v as bf16 high / low parts
     int32_t off_w, off_tok, tok_bytes, n_stages;               // ring of job buffers: weight tiles, token rows
+    int32_t w_bytes;                                           // general kernel: bytes of a stage's weight tile
     int32_t moff_perm, moff_udesc, moff_uperm;                 // word offsets: perm, unit records, unit row ids
     FusedItem item[MAX_ITEMS];
 };
@@ -122,7 +124,7 @@ lora_status_t build_fused_maps(lora_pool_t *pool) {
         for (int i = 0; i < 8; ++i) {
             const int rows = 8 * (i + 1);
             if (rows > ((pool->r_max + 7) & ~7)) break;   // no slot holds that many rank rows
-            const int blocks = rows <= 16 ? 4 : rows <= 32 ? 2 : 1;   // chunk width 256 / 128 / 64
+            const int blocks = rows <= 32 ? 4 : 2;   // chunk width 256 columns up to 32 rank rows, 128 above
             if (!weight_map(fn, &maps[(size_t)t * MAPS_PER_TARGET + i], w + tv.off_a, tv.d_in, pool->r_max,
                             pool->num_slots, pool->slot_stride, rows, blocks) ||
                 !weight_map(fn, &maps[(size_t)t * MAPS_PER_TARGET + 8 + i], w + tv.off_b, tv.d_out, pool->r_max,
@@ -158,7 +160,9 @@ static lora_status_t launch_h(lora_pool_t *pool, FusedParams &P, int32_t C, cons
     P.off_vh = o;     o += mrows * gen::PV * 2;
     P.off_vl = o;     o += mrows * gen::PV * 2;
     o = (o + 1023) & ~1023;
-    P.off_w = o;      o += S * W_BYTES;
+    // a pool that has never held a rank above 16 needs only 8 KB tiles (16 rank rows x 256 columns)
+    P.w_bytes = RPmax <= 16 ? W_BYTES : GEN_W_BYTES;
+    P.off_w = o;      o += S * P.w_bytes;
     P.tok_bytes = mrows * TOK_PITCH * 2;
     P.off_tok = o;    o += S * P.tok_bytes;
     P.n_stages = S;
@@ -258,7 +262,11 @@ lora_status_t launch_fused_items(lora_pool_t *pool, const ApplyParams *items, in
     // cluster size: as wide a split as the narrowest projection of the launch supports
     int32_t C = pool->tuning[1];
     if (C != 1 && C != 2 && C != 4 && C != 8) {
-        C = 8;
+        // Eight blocks per unit shorten a unit's chain, four leave twice as many clusters for a
+        // batch with several units per cluster: a long prefill-type batch that keeps all its tiles
+        // here has hundreds of 16-row units (mixed chunked prefill: 84 us with 4, 91 us with 8);
+        // what the tensor-core kernels leave over is a handful of units (prefill: 322 us with 8, 347 with 4).
+        C = (tile_m > 8 && A0.T >= 1024 && P.path_filter == 0) ? 4 : 8;
         for (int32_t i = 0; i < n_items; ++i)
             while (C > 1 && (items[i].tv.d_in / C < 256 || items[i].tv.d_out / C < 128)) C >>= 1;
     }

@@ -11,8 +11,8 @@
 // A job is one column chunk: the rank rows of A_i (or B_i) by ONE tiled bulk copy (TMA, 128-byte
 // swizzle), the unit's rows of x (or y_base) by one bulk copy per row, and a 16-byte header (kind,
 // first / last chunk of its unit, columns, unit entry).  The four consumer warps hold no control
-// logic: they follow the headers.  The chunk width shrinks as the rank grows (256 / 128 / 64 columns
-// for ranks <= 16 / 32 / 64), so a stage is the same size for every rank.
+// logic: they follow the headers.  A chunk is 256 columns wide up to rank 32 and 128 above, so a
+// weight tile is at most 16 KB and a stage has one size for every rank.
 //   shrink   bf16 MMA (m16n8k16), fp32 accumulators carried across a unit's chunks in registers;
 //   exchange every block keeps its partial in its own shared memory and tells the cluster; every
 //            block then reads all partials (distributed shared memory) and sums them in block order;
@@ -40,6 +40,9 @@ constexpr int UNIT_ENTRIES = 8;
 constexpr int UNIT_BYTES = 96;
 constexpr int PV = 72;           // elements between rows of the bf16 copies of v
 static_assert(SM_UNIT + UNIT_ENTRIES * UNIT_BYTES <= SM_HEADER, "fixed part fits before the carved-up buffers");
+
+// columns of a job for rank bucket 16 << sh: the weight tile is at most 16 KB
+__host__ __device__ constexpr int chunk_cols(int sh) { return sh == 2 ? 128 : 256; }
 
 enum { J_SHRINK = 1, J_FIRST = 2, J_LAST = 4, J_END = 8 /* no data, stream over */,
        J_FINAL = 16 /* last job of the stream */, J_COPY = 32 /* y_base -> y for one row */ };
@@ -85,10 +88,10 @@ __device__ __forceinline__ PUnit p_decode(const FusedParams &P, uint32_t crank, 
             !(P.path_filter && contiguous && tile_rows >= P.path_filter);
     u.copy = !P.meta && rec.x == -1 && !it.in_place;
     u.sh = u.rank <= 16 ? 0 : u.rank <= 32 ? 1 : 2;
-    const int32_t cw = 256 >> u.sh;
+    const int32_t cw = chunk_cols(u.sh);
     // at least one job per phase: a block without columns still takes part in the exchange
-    u.na = max(1, (u.a_hi - u.a_lo + cw - 1) >> (8 - u.sh));
-    u.nb = max(1, (u.b_hi - u.b_lo + cw - 1) >> (8 - u.sh));
+    u.na = max(1, (u.a_hi - u.a_lo + cw - 1) / cw);
+    u.nb = max(1, (u.b_hi - u.b_lo + cw - 1) / cw);
     return u;
 }
 
@@ -125,7 +128,7 @@ __device__ __forceinline__ void p_request(const FusedParams &P, unsigned char *s
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + SM_FULL) + st;
     const bool shrink = j < un.na;
     const int32_t c = shrink ? j : j - un.na;
-    const int32_t cw = 256 >> un.sh;
+    const int32_t cw = chunk_cols(un.sh);
     const int32_t col0 = (shrink ? un.a_lo : un.b_lo) + c * cw;   // a multiple of 64
     const int32_t ncols = max(0, min(cw, (shrink ? un.a_hi : un.b_hi) - col0));
     if (lane == 0 && mode != 2) {
@@ -137,7 +140,7 @@ __device__ __forceinline__ void p_request(const FusedParams &P, unsigned char *s
             const CUtensorMap *map = P.maps + it.map_base + (shrink ? 0 : 8) + (un.rb >> 3) - 1;
             // the tile load always delivers its whole box: rb rows of cw columns
             mbar_expect_tx(full, (uint32_t)un.rb * (uint32_t)cw * 2u + (uint32_t)un.rows * (uint32_t)ncols * 2u);
-            tma_load_4d(smem + P.off_w + st * W_BYTES, map, 0, 0, col0 >> 6, un.slot, full);
+            tma_load_4d(smem + P.off_w + st * P.w_bytes, map, 0, 0, col0 >> 6, un.slot, full);
         } else {
             mbar_arrive(full);   // header only
         }
@@ -289,7 +292,7 @@ struct CLane {
 // One shrink chunk: acc += x[rows, chunk] . A_i[chunk, 16 ranks of this warp].  RP: rank bucket; H: 1
 // when a unit holds at most 8 rows, 2 when rows 8..15 can be occupied.  The four warps split the
 // rank tiles WN ways and the chunk's 64-column blocks WK ways: every warp owns two rank tiles of 8
-// and one column block.  Operand fragments come by ldmatrix; lane l names row (l & 7) of 8x8 matrix
+// and every WK-th column block.  Operand fragments come by ldmatrix; lane l names row (l & 7) of 8x8 matrix
 // (l >> 3):
 //   weights: (tile 2wn, k 0-7) (tile 2wn, k 8-15) (tile 2wn+1, k 0-7) (tile 2wn+1, k 8-15); rank row
 //            n sits at n * 128 bytes of the column block, its 16-byte chunk c at ((c ^ (n & 7)) << 4);
@@ -299,30 +302,34 @@ template <int RP, int H>
 __device__ __forceinline__ void shrink_job(const CLane &L, uint32_t w_stage, uint32_t t_stage, int32_t ncols,
                                            uint32_t blk_bytes, float (&acc)[2][4]) {
     constexpr int WN = RP / 16, WK = 4 / WN;
+    constexpr int NB = chunk_cols(RP == 16 ? 0 : RP == 32 ? 1 : 2) / 64;   // column blocks of a job
     constexpr bool hi_rows = H == 2;
     const int wk = L.warp % WK, wn = L.warp / WK;
-    const int32_t nc = ncols - wk * 64;   // columns of this warp's block
-    if (nc <= 0) return;
-    const uint32_t As = w_stage + (uint32_t)wk * blk_bytes + (uint32_t)(16 * wn + 8 * (L.mi >> 1) + L.r) * 128u +
-                        (uint32_t)(((L.mi & 1) ^ L.r) << 4);
-    const uint32_t X = t_stage + (uint32_t)wk * 128u +
-                       (hi_rows ? (uint32_t)(((L.mi & 1) * 8 + L.r) * TOK_PITCH + (L.mi >> 1) * 8) * 2u
-                                : (uint32_t)(L.r * TOK_PITCH + (L.mi & 1) * 8) * 2u);
+    const uint32_t w_lane = (uint32_t)(16 * wn + 8 * (L.mi >> 1) + L.r) * 128u + (uint32_t)(((L.mi & 1) ^ L.r) << 4);
+    const uint32_t x_lane = hi_rows ? (uint32_t)(((L.mi & 1) * 8 + L.r) * TOK_PITCH + (L.mi >> 1) * 8) * 2u
+                                    : (uint32_t)(L.r * TOK_PITCH + (L.mi & 1) * 8) * 2u;
 #pragma unroll
-    for (int ks = 0; ks < 64; ks += 16) {
-        if (ks < nc) {   // the ragged end of a slice: columns past it hold neither x nor these weights
-            const bool full = nc - ks >= 16;   // else only 8 columns are left
-            uint32_t a[4], bw[4];
-            if (hi_rows) {
-                ldmatrix_x4(a, X + ks * 2);
-            } else {
-                ldmatrix_x2(a[0], a[2], X + ks * 2);
-                a[1] = a[3] = 0u;
+    for (int cb = wk; cb < NB; cb += WK) {   // this warp's column blocks of the job
+        const int32_t nc = ncols - cb * 64;
+        if (nc <= 0) break;
+        const uint32_t As = w_stage + (uint32_t)cb * blk_bytes + w_lane;
+        const uint32_t X = t_stage + (uint32_t)cb * 128u + x_lane;
+#pragma unroll
+        for (int ks = 0; ks < 64; ks += 16) {
+            if (ks < nc) {   // the ragged end of a slice: columns past it hold neither x nor these weights
+                const bool full = nc - ks >= 16;   // else only 8 columns are left
+                uint32_t a[4], bw[4];
+                if (hi_rows) {
+                    ldmatrix_x4(a, X + ks * 2);
+                } else {
+                    ldmatrix_x2(a[0], a[2], X + ks * 2);
+                    a[1] = a[3] = 0u;
+                }
+                ldmatrix_x4(bw, As ^ (uint32_t)((ks >> 3) << 4));
+                if (!full) a[2] = a[3] = bw[1] = bw[3] = 0u;
+                mma16816(acc[0], a, bw[0], bw[1]);
+                mma16816(acc[1], a, bw[2], bw[3]);
             }
-            ldmatrix_x4(bw, As ^ (uint32_t)((ks >> 3) << 4));
-            if (!full) a[2] = a[3] = bw[1] = bw[3] = 0u;
-            mma16816(acc[0], a, bw[0], bw[1]);
-            mma16816(acc[1], a, bw[2], bw[3]);
         }
     }
 }
@@ -342,7 +349,7 @@ struct XUnit {
 template <int RP, int H>
 __device__ __forceinline__ void expand_job(const CLane &L, uint32_t w_stage, uint32_t t_stage, uint32_t vh,
                                            uint32_t vl, int32_t ncols, int32_t c, const XUnit &xu) {
-    constexpr int CW = 4096 / RP, NW = CW / 4, NP = NW / 16, KT = RP / 16;
+    constexpr int CW = chunk_cols(RP == 16 ? 0 : RP == 32 ? 1 : 2), NW = CW / 4, NP = NW / 16, KT = RP / 16;
     constexpr bool hi_rows = H == 2;
     const int32_t nc = ncols - L.warp * NW;   // columns of this warp's share
     if (nc <= 0) return;
@@ -458,7 +465,7 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
         }
         const int4 job = *reinterpret_cast<const int4 *>(smem + SM_JOB + 16 * st);
         if (job.x & J_END) break;
-        const uint32_t w_stage = w_base + st * W_BYTES, t_stage = t_base + st * P.tok_bytes;
+        const uint32_t w_stage = w_base + st * P.w_bytes, t_stage = t_base + st * P.tok_bytes;
         if (job.x & J_COPY) {
             // per-token mode: row job.z of projection job.y takes no adapter
             const FusedItem &it = P.item[job.y];
@@ -559,7 +566,7 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
                 if (tid < (int)csize) mbar_arrive_peer(reinterpret_cast<uint64_t *>(smem + SM_YB) + b, (uint32_t)tid);
                 ++kr;
                 const FusedItem &it = P.item[ue->item];
-                const int NW = 64 >> sh;
+                const int NW = chunk_cols(sh) / 4;
                 xu.row0 = L.g < rows;
                 xu.row1 = H == 2 && L.g + 8 < rows;
                 xu.y0 = it.y + (int64_t)(xu.row0 ? ue->rowid[L.g] : 0) * it.ldy + ue->b_lo + L.warp * NW + 2 * L.t;
@@ -600,12 +607,27 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
             if (!meet()) break;
             if (tid < rows) rowidx[tid] = __ldg(P.meta + P.moff_perm + n_active + first + tid);
             if (!meet()) break;
+            // the chunk's rows as one index space (row, 16-byte vector of this block's share), four
+            // independent loads in flight per thread
             const int32_t vecs = it.d_out / 8;
-            for (int32_t m = 0; m < rows; ++m) {
-                const __nv_bfloat16 *src = it.yb + (int64_t)rowidx[m] * it.ldyb;
-                __nv_bfloat16 *dst = it.y + (int64_t)rowidx[m] * it.ldy;
-                for (int32_t v = (int32_t)crank * FT + tid; v < vecs; v += (int32_t)csize * FT)
-                    reinterpret_cast<uint4 *>(dst)[v] = ldg16(src + (int64_t)v * 8);
+            const int32_t per_blk = (vecs + (int32_t)csize - 1) / (int32_t)csize;
+            const int32_t v_lo = (int32_t)crank * per_blk, v_n = max(0, min(per_blk, vecs - v_lo));
+            const int32_t total = rows * v_n;
+            for (int32_t i0 = tid; i0 < total; i0 += 4 * FT) {
+                uint4 val[4];
+                int64_t off[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int32_t i = i0 + q * FT;
+                    const int32_t m = i < total ? i / v_n : 0, v = i < total ? v_lo + i - m * v_n : 0;
+                    off[q] = (int64_t)rowidx[m];
+                    val[q] = make_uint4(0, 0, 0, 0);
+                    if (i < total) val[q] = ldg16(it.yb + off[q] * it.ldyb + (int64_t)v * 8);
+                    off[q] = off[q] * it.ldy + (int64_t)v * 8;
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (i0 + q * FT < total) *reinterpret_cast<uint4 *>(it.y + off[q]) = val[q];
             }
         }
     }
