@@ -8,6 +8,9 @@
 
 namespace lora {
 
+constexpr uint32_t WAIT_HINT_NS = 2000;      // how long one poll of a barrier may sleep
+constexpr uint32_t WAIT_POLLS = 1u << 17;    // polls before a wait is given up
+
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
     return (uint32_t)__cvta_generic_to_shared(p);
 }
@@ -34,16 +37,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(WAIT_HINT_NS)
         : "memory");
     return ok != 0;
 }
-// bounded wait: gives up after a fixed number of polls instead of spinning for ever
+// bounded wait: gives up after a fixed number of polls instead of spinning for ever.  Every poll
+// may sleep in the hardware for up to WAIT_HINT_NS (it wakes as soon as the phase completes), so a
+// waiting warp issues few instructions; the bound is WAIT_POLLS polls, a fraction of a second.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
-    for (uint32_t i = 0; i < (1u << 20); ++i)
+    for (uint32_t i = 0; i < WAIT_POLLS; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -92,14 +97,14 @@ __device__ __forceinline__ void mbar_arrive_peer(uint64_t *local_bar, uint32_t r
 }
 // bounded wait on this block's mbarrier for arrivals from the whole cluster (acquire at cluster scope)
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity) {
-    for (uint32_t i = 0; i < (1u << 20); ++i) {
+    for (uint32_t i = 0; i < WAIT_POLLS; ++i) {
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(ok)
-            : "r"(smem_u32(bar)), "r"(parity)
+            : "r"(smem_u32(bar)), "r"(parity), "r"(WAIT_HINT_NS)
             : "memory");
         if (ok) return true;
     }
