@@ -433,14 +433,12 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
 #pragma unroll
                 for (int np = 0; np < 4; ++np) {
                     float ex[2][4];
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) ex[j][0] = ex[j][1] = ex[j][2] = ex[j][3] = 0.0f;
                     uint32_t bb[4];
                     ldmatrix_x4_trans(bb, Bs ^ (uint32_t)(np << 5));
                     if (!upper) bb[1] = bb[3] = 0u;
-                    mma16816(ex[0], ah, bb[0], bb[1]);
+                    mma16816_first(ex[0], ah, bb[0], bb[1]);
+                    mma16816_first(ex[1], ah, bb[2], bb[3]);
                     mma16816(ex[0], al, bb[0], bb[1]);
-                    mma16816(ex[1], ah, bb[2], bb[3]);
                     mma16816(ex[1], al, bb[2], bb[3]);
                     // epilogue straight from the accumulator layout: each lane owns two adjacent
                     // columns of row g per column tile; a quad covers 16 contiguous bytes
