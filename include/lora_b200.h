@@ -175,7 +175,8 @@ lora_status_t lora_pool_selftest_wait_expiry(lora_pool_t *pool, int32_t polls, i
  *   key 3  fused kernel: upper bound on the clusters in the grid
  *   key 4  tensor-core kernels of lora_sgmv_apply: 1 = never, 2 = whenever they apply
  *   key 5  fused kernel: stages of the shared-memory ring (2 .. 4)
- *   key 6  (unused)
+ *   key 6  lora_sgmv_apply: 1 = the tiles the tensor-core kernels leave over run after them on the
+ *          caller's stream, not beside them on the pool's own stream
  *   key 7  segment builder: 1 = one warp per slot also for long batches
  *   key 8  (unused)
  *   key 9  fused kernel: share (1 .. 99 %) of the resident clusters one launch may take
@@ -356,7 +357,11 @@ lora_status_t lora_bgmv_apply_static(lora_pool_t *pool, int32_t target,
 /* Prefill / chunked-prefill batches.  meta_dev: metadata built for this batch (any tile_m).
  * With tile_m = 128 and a batch of at least 4096 tokens, tiles that are runs of 32 .. 128
  * consecutive tokens take the tcgen05 kernels (split-K partials in `workspace`); every other tile,
- * and every tile of a shorter batch, takes the fused kernel that also serves lora_bgmv_apply. */
+ * and every tile of a shorter batch, takes the fused kernel that also serves lora_bgmv_apply.
+ * When both kinds are present the fused kernel runs on a stream the pool owns, forked from
+ * `stream` by an event at the call and joined back into it before the call returns, so work
+ * enqueued on `stream` afterwards is ordered behind all of it (this also holds inside a stream
+ * capture: the pool's stream joins the capture and leaves it within the call). */
 lora_status_t lora_sgmv_apply(lora_pool_t *pool, int32_t target,
                               const void *x, int64_t ldx,
                               const void *y_base, int64_t ldyb,

@@ -54,6 +54,7 @@ void fill_apply_params(lora_pool_t *pool, ApplyParams &P, int32_t target, const 
     P.stage_bytes = P.n_stages = 0;
     P.moff_perm = P.moff_udesc = P.moff_uperm = 0;
     P.path_filter = 0;
+    P.no_pdl = 0;
     P.early = 0;
     P.push = 0;
 }
@@ -69,13 +70,41 @@ static lora_status_t apply_common(lora_pool_t *pool, int32_t target, const void 
     if (!workspace || workspace_bytes < (size_t)T * P.RS * sizeof(float))
         return LORA_ERR_BUFFER_TOO_SMALL;
     if (pool->tuning[0] == 1) return launch_twophase(pool, P, workspace, workspace_bytes, stream);
-    // prefill batches: full tiles of 128 consecutive tokens go to the tensor-core kernels
-    // (tuning key 4 = 1 keeps everything on the fused kernel)
+    // prefill batches: runs of consecutive tokens go to the tensor-core kernels (tuning key 4 = 1
+    // keeps everything on the fused kernel)
     if (use_tc && pool->tuning[4] != 1) {
-        bool handled = false;
-        lora_status_t s = launch_tc_long_tiles(pool, P, workspace, workspace_bytes, stream, &handled);
+        bool applies = false;
+        lora_status_t s = launch_tc_long_tiles(pool, P, workspace, workspace_bytes, stream, &applies, true);
         if (s != LORA_OK) return s;
-        P.path_filter = handled ? 32 : 0;   // runs of >= 32 consecutive tokens were taken there
+        if (applies) {
+            // The tiles those kernels leave over (short, ragged or scattered ones: a handful of
+            // units whose chains take tens of microseconds but move few bytes) run beside them on
+            // the pool's own stream, forked from and joined back into the caller's stream; the two
+            // parts write disjoint rows of y.  Tuning key 6 = 1: one after the other.
+            ApplyParams rest = P;
+            rest.path_filter = 32;   // runs of >= 32 consecutive tokens are taken by the other path
+            const bool beside = pool->side_stream && pool->tuning[6] != 1;
+            lora_status_t s_rest = LORA_OK;
+            if (beside) {
+                LORA_CUDA_TRY(cudaEventRecord(pool->ev_fork, stream));
+                LORA_CUDA_TRY(cudaStreamWaitEvent(pool->side_stream, pool->ev_fork, 0));
+                rest.no_pdl = 1;
+                s_rest = launch_fused(pool, rest, pool->side_stream);
+                cudaError_t e = cudaEventRecord(pool->ev_join, pool->side_stream);
+                if (e != cudaSuccess && s_rest == LORA_OK) s_rest = cuda_fail(e);
+            }
+            bool handled = false;
+            s = launch_tc_long_tiles(pool, P, workspace, workspace_bytes, stream, &handled, false);
+            if (beside) {
+                // the join is made whatever happened above, so a capture of the caller's stream
+                // never ends with the pool's stream still forked from it
+                cudaError_t e = cudaStreamWaitEvent(stream, pool->ev_join, 0);
+                if (e != cudaSuccess && s == LORA_OK) s = cuda_fail(e);
+            } else if (s == LORA_OK) {
+                s_rest = launch_fused(pool, rest, stream);
+            }
+            return s != LORA_OK ? s : s_rest;
+        }
     }
     return launch_fused(pool, P, stream);
 }

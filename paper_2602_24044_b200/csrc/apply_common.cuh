@@ -30,6 +30,7 @@ struct ApplyParams {
     int32_t push;              // fused path: block partials are pushed to all blocks of the cluster (small units)
     int32_t early;             // the unit records and the pool may be read before the preceding kernel has finished
     int32_t path_filter;       // 0 = every unit; else skip runs of at least this many consecutive tokens
+    int32_t no_pdl;            // 1 = plain launch (the kernel does not follow a kernel of its own stream)
 };
 
 struct Tile {
@@ -141,7 +142,8 @@ lora_status_t launch_fused_items(lora_pool_t *pool, const ApplyParams *items, in
                                  cudaStream_t stream);
 lora_status_t build_fused_maps(lora_pool_t *pool);
 lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, void *workspace,
-                                   size_t workspace_bytes, cudaStream_t stream, bool *handled);
+                                   size_t workspace_bytes, cudaStream_t stream, bool *handled,
+                                   bool check_only);
 lora_status_t launch_build_segments(lora_pool_t *pool, const int32_t *slot_idx_dev, int32_t T,
                                     int32_t tile_m, int32_t long_min, void *meta_dev,
                                     cudaStream_t stream);

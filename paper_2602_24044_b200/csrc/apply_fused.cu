@@ -62,6 +62,7 @@ struct FusedParams {
     int32_t early;             // the unit records and the pool may be read before the preceding kernel has finished
     int32_t push;              // block partials are pushed to all blocks of the cluster (small units)
     int32_t path_filter;       // 0 = every unit; else skip runs of at least this many consecutive tokens
+    int32_t no_pdl;            // host side only: launch without the programmatic-launch attribute
     int32_t late_trigger;      // decode kernel: let the successor in only once this kernel's blocks are set up
     int32_t copy_idle;         // some projection is out of place: rows without adapter are copied
     int32_t off_part, off_vpart, vbuf_bytes, off_vh, off_vl;   // warp partials, exchange buffers (x2), v as bf16 high / low parts
@@ -196,10 +197,10 @@ static lora_status_t launch_h(lora_pool_t *pool, FusedParams &P, int32_t C, cons
     // has already been read by an earlier apply: that apply was fully ordered behind the build, so
     // the table is complete before this kernel can start.
     const bool fresh = meta_key ? pool->take_fresh(meta_key) : true;
-    P.early = (meta_key && !fresh && pool->tuning[2] != 2) ? 1 : 0;
+    P.early = (meta_key && !fresh && pool->tuning[2] != 2 && !P.no_pdl) ? 1 : 0;
     // Without `early` the attribute still lets the blocks become resident and set up their shared
     // memory while the kernel before them drains; they read nothing until it has completed.
-    const unsigned n_attrs = pool->tuning[2] != 2 ? 2 : 1;
+    const unsigned n_attrs = (pool->tuning[2] != 2 && !P.no_pdl) ? 2 : 1;
 
     // Grid: no more clusters than can be resident at once (each loops over its units), so no
     // cluster of an over-sized grid waits for a slot only to find that its unit does not exist.
@@ -248,6 +249,7 @@ lora_status_t launch_fused_items(lora_pool_t *pool, const ApplyParams *items, in
     P.T = A0.T;
     P.n_items = n_items;
     P.path_filter = A0.path_filter;
+    P.no_pdl = A0.no_pdl;
     const int32_t tile_m = A0.meta ? A0.tile_m : 1;
     P.units_cap = A0.T;
     if (A0.meta) {

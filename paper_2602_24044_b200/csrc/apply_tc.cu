@@ -156,8 +156,7 @@ __host__ __device__ constexpr uint32_t instr_desc(uint32_t M, uint32_t N, uint32
 }
 }  // namespace tc
 
-constexpr int TC_THREADS = 128;
-constexpr int TCX_THREADS = 160;   // expand: four epilogue warps and one warp that issues copies and MMAs
+constexpr int TCX_THREADS = 192;   // expand: four epilogue warps, one warp that issues MMAs, one that issues copies
 constexpr int TC_ROWS = 128;       // rows of a long tile
 constexpr int SH_STAGES = 4;       // shrink: ring of (x tile, A tile) stages
 constexpr int XT_BYTES = TC_ROWS * 128;   // 128 rows x 64 bf16
@@ -166,8 +165,9 @@ struct TcParams {
     PoolView pool;
     TargetView tv;
     const int32_t *meta;
-    float *ws;              // [KS][T][RS] fp32 partial v
-    int32_t T, RS, KS, NS;
+    float *ws;              // [KS][T][RS] fp32 partial v: one slab per piece of a tile
+    int32_t T, RS, KS, NS;  // KS: slabs the workspace holds
+    int32_t shrink_grid;    // blocks of the shrink launch (fixes how the walk is cut into pieces)
     int32_t moff_perm, moff_desc;
     int32_t target_rows;    // r_max: rows of a slot's matrices
     __nv_bfloat16 *y;       // output, for tiles with fewer than 128 rows (stored row by row)
@@ -245,8 +245,44 @@ tc_worklist_kernel(const TcParams P) {
 // ---------------------------------------------------------------------------------------------
 // shrink
 // ---------------------------------------------------------------------------------------------
+// The shrink walks the (long tile, 64-column K-block) pairs of the batch in tile order.  The walk is
+// cut into equal spans, one per block of a grid that fills the GPU exactly once, so every block
+// streams the same number of bytes whatever the number of long tiles is.  A span may end inside a
+// tile: the part of tile t that block b computes is the tile's "piece" b - first_block(t), and its
+// fp32 partial goes to slab [piece] of the workspace; the expand adds a tile's pieces in order.
+struct ShrinkSplit {
+    int64_t total;     // K-blocks of all long tiles
+    int32_t nkb;       // K-blocks of one tile
+    int32_t span;      // K-blocks per block
+};
+// slabs: partial slabs the workspace holds (a tile must not be cut into more pieces than that)
+__host__ __device__ inline ShrinkSplit shrink_split(int32_t n_long, int32_t d_in, int32_t slabs, int32_t grid) {
+    ShrinkSplit sp;
+    sp.nkb = (d_in + 63) / 64;
+    sp.total = (int64_t)n_long * sp.nkb;
+    int64_t span = (sp.total + grid - 1) / grid;
+    if (slabs <= 1) {
+        span = ((span + sp.nkb - 1) / sp.nkb) * sp.nkb;          // whole tiles only
+    } else {
+        const int64_t least = (sp.nkb + slabs - 2) / (slabs - 1);   // at most slabs pieces per tile
+        if (span < least) span = least;
+    }
+    if (span < 1) span = 1;
+    sp.span = (int32_t)span;
+    return sp;
+}
+// pieces of tile entry t: blocks first .. last of the walk touch it
+__host__ __device__ inline int32_t first_block_of(const ShrinkSplit &sp, int32_t t) {
+    return (int32_t)(((int64_t)t * sp.nkb) / sp.span);
+}
+__host__ __device__ inline int32_t last_block_of(const ShrinkSplit &sp, int32_t t) {
+    return (int32_t)((((int64_t)t + 1) * sp.nkb - 1) / sp.span);
+}
+
+constexpr int TCS_THREADS = 192;   // shrink: four warps that write partials, one MMA thread, one loading thread
+
 template <int RP>
-__global__ void __launch_bounds__(TC_THREADS)
+__global__ void __launch_bounds__(TCS_THREADS)
 tc_shrink_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_x,
                  const __grid_constant__ CUtensorMap map_a) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -255,28 +291,30 @@ tc_shrink_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_x,
         ((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     constexpr int AT_BYTES = RP * 128;               // RP rank rows x 64 bf16
     constexpr int STAGE = XT_BYTES + ((AT_BYTES + 1023) & ~1023);
-    constexpr uint32_t TMEM_COLS = RP < 32 ? 32 : RP;
+    constexpr uint32_t ACC = RP < 32 ? 32 : RP;      // columns of one accumulator
+    constexpr uint32_t TMEM_COLS = 2 * ACC;          // two accumulators: a piece is written out while the next one runs
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + SH_STAGES * STAGE);
     uint64_t *empty = full + SH_STAGES;
-    uint64_t *done = empty + SH_STAGES;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(done + 1);
+    uint64_t *done = empty + SH_STAGES;              // [2] all MMAs of a piece have completed
+    uint64_t *acc_free = done + 2;                   // [2] the accumulator has been read out
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_free + 2);
+    volatile int32_t *failed = reinterpret_cast<volatile int32_t *>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const LongTile lt = long_tile(P, blockIdx.x);
-    if (!lt.ok) return;
-    const int32_t ks = blockIdx.y;
-    // K-blocks of 64 columns owned by this block
-    const int32_t nkb_all = (P.tv.d_in + 63) / 64;
-    const int32_t per = (nkb_all + P.KS - 1) / P.KS;
-    const int32_t kb0 = min(ks * per, nkb_all), kb1 = min(kb0 + per, nkb_all);
-    const int32_t nkb = kb1 - kb0;
+    const int32_t n_long = P.list[0];
+    if (n_long <= 0) return;
+    const ShrinkSplit sp = shrink_split(n_long, P.tv.d_in, P.KS, (int32_t)gridDim.x);
+    const int64_t g0 = (int64_t)blockIdx.x * sp.span;
+    const int64_t g1 = min(g0 + (int64_t)sp.span, sp.total);
+    if (g0 >= g1) return;
 
     if (tid == 0) {
         for (int s = 0; s < SH_STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
-        tc::mbar_init(done, 1);
+        for (int s = 0; s < 2; ++s) { tc::mbar_init(&done[s], 1); tc::mbar_init(&acc_free[s], 128); }
+        *failed = 0;
         tc::fence_mbar_init();
     }
-    if (warp == 0) {
+    if (warp == 4) {
         tc::tmem_alloc(tmem_slot, TMEM_COLS);
         tc::tmem_relinquish();
     }
@@ -284,78 +322,114 @@ tc_shrink_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_x,
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    bool ok = true;
 
-    // Two single-thread roles in different warps: one requests tiles (it alone waits for a stage
-    // to be read out before refilling it), one issues the MMAs (it only ever waits for data).
-    int32_t issued = 0;   // tiles requested by the loading thread
-    if (tid == 32 && nkb > 0) {
-        for (int32_t i = 0; i < nkb && ok; ++i, ++issued) {
-            const int s = i % SH_STAGES;
-            if (i >= SH_STAGES) ok = tc::mbar_wait(&empty[s], (uint32_t)(i / SH_STAGES - 1) & 1u);
-            if (!ok) break;
-            unsigned char *st = smem + s * STAGE;
-            tc::mbar_expect_tx(&full[s], XT_BYTES + AT_BYTES);
-            tc::tma_load_2d(st, &map_x, (kb0 + i) * 64, lt.t0, &full[s]);
-            tc::tma_load_3d(st + XT_BYTES, &map_a, (kb0 + i) * 64, 0, lt.slot, &full[s]);
-        }
-    }
-    if (tid == 0 && nkb > 0) {
-        constexpr uint32_t IDESC = tc::instr_desc(128, RP, 0, 0);
-        for (int32_t i = 0; i < nkb && ok; ++i) {
-            const int s = i % SH_STAGES;
-            const uint32_t ph = (uint32_t)(i / SH_STAGES) & 1u;
-            ok = tc::mbar_wait(&full[s], ph);
-            if (!ok) break;
-            tc::tc_fence_after();
-            const uint32_t xa = tc::smem_u32(smem + s * STAGE), aa = xa + XT_BYTES;
-#pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4) {   // four K = 16 steps inside the 128-byte swizzle atom
-                const uint64_t ad = tc::smem_desc(xa + k4 * 32, 16, 1024, tc::LAYOUT_SW128);
-                const uint64_t bd = tc::smem_desc(aa + k4 * 32, 16, 1024, tc::LAYOUT_SW128);
-                tc::umma(tmem, ad, bd, IDESC, (i > 0 || k4 > 0) ? 1u : 0u);
+    if (warp == 5) {
+        // ---- loading thread: requests the (x tile, A tile) pairs of the whole span in order; it
+        // alone waits for a stage to be read out before refilling it ----------------------------
+        if (lane == 0) {
+            int32_t issued = 0;
+            bool ok = true;
+            int32_t t = (int32_t)(g0 / sp.nkb), kb = (int32_t)(g0 % sp.nkb);
+            LongTile lt = long_tile(P, t);
+            for (int64_t g = g0; g < g1 && ok; ++g) {
+                const int s = issued % SH_STAGES;
+                if (issued >= SH_STAGES) ok = tc::mbar_wait(&empty[s], (uint32_t)(issued / SH_STAGES - 1) & 1u);
+                if (!ok || *failed || !lt.ok) { ok = false; break; }
+                unsigned char *st = smem + s * STAGE;
+                tc::mbar_expect_tx(&full[s], XT_BYTES + AT_BYTES);
+                tc::tma_load_2d(st, &map_x, kb * 64, lt.t0, &full[s]);
+                tc::tma_load_3d(st + XT_BYTES, &map_a, kb * 64, 0, lt.slot, &full[s]);
+                ++issued;
+                if (++kb == sp.nkb && g + 1 < g1) {
+                    kb = 0;
+                    lt = long_tile(P, ++t);
+                }
             }
-            tc::umma_commit(&empty[s]);   // the stage may be refilled once these MMAs have read it
-        }
-        tc::umma_commit(done);
-    }
-    __syncwarp();
-    if (nkb > 0) {
-        if (!tc::mbar_wait(done, 0)) ok = false;
-    }
-    tc::tc_fence_after();
-    // accumulator -> fp32 partial in the workspace (thread = row of the tile)
-    const int32_t m = warp * 32 + lane;
-    float *dst = P.ws + ((int64_t)ks * P.T + lt.row0 + m) * P.RS;
-    const bool all_ok = __syncthreads_and(ok ? 1 : 0) != 0;
-    if (all_ok) {
-#pragma unroll
-        for (int c = 0; c < RP; c += 16) {
-            uint32_t r[16];
-            if (nkb > 0) {      // whole warps take part in the tensor-memory load
-                tc::tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + c, r);
-                tc::tmem_ld_wait();
-            } else {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) r[i] = 0u;
-            }
-            if (m < lt.rows) {  // rows past a short tile's end belong to other tiles
-#pragma unroll
-                for (int i = 0; i < 16; i += 4)
-                    *reinterpret_cast<uint4 *>(dst + c + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+            if (!ok) {
+                *failed = 1;
+                // copies still on their way into this block's shared memory must land before it
+                // leaves: the most recent request of every stage is waited for (bounded)
+                for (int32_t q = max(issued - SH_STAGES, 0); q < issued; ++q)
+                    tc::mbar_wait(&full[q % SH_STAGES], (uint32_t)(q / SH_STAGES) & 1u);
             }
         }
+        __syncwarp();
+    } else if (warp == 4) {
+        // ---- MMA thread: it only ever waits for data (and, from the third piece on, for the
+        // accumulator it reuses) -----------------------------------------------------------------
+        if (lane == 0) {
+            constexpr uint32_t IDESC = tc::instr_desc(128, RP, 0, 0);
+            int32_t i = 0, piece = 0;
+            bool ok = true;
+            for (int64_t g = g0; g < g1 && ok; ++piece) {
+                const int32_t kb = (int32_t)(g % sp.nkb);
+                const int32_t len = (int32_t)min((int64_t)(sp.nkb - kb), g1 - g);
+                const uint32_t acc = tmem + (uint32_t)(piece & 1) * ACC;
+                if (piece >= 2) ok = tc::mbar_wait(&acc_free[piece & 1], (uint32_t)(piece / 2 - 1) & 1u);
+                tc::tc_fence_after();
+                for (int32_t k = 0; k < len && ok; ++k, ++i) {
+                    const int s = i % SH_STAGES;
+                    ok = !*failed && tc::mbar_wait(&full[s], (uint32_t)(i / SH_STAGES) & 1u);
+                    if (!ok) break;
+                    tc::tc_fence_after();
+                    const uint32_t xa = tc::smem_u32(smem + s * STAGE), aa = xa + XT_BYTES;
+#pragma unroll
+                    for (int k4 = 0; k4 < 4; ++k4) {   // four K = 16 steps inside the 128-byte swizzle atom
+                        const uint64_t ad = tc::smem_desc(xa + k4 * 32, 16, 1024, tc::LAYOUT_SW128);
+                        const uint64_t bd = tc::smem_desc(aa + k4 * 32, 16, 1024, tc::LAYOUT_SW128);
+                        tc::umma(acc, ad, bd, IDESC, (k > 0 || k4 > 0) ? 1u : 0u);
+                    }
+                    tc::umma_commit(&empty[s]);   // the stage may be refilled once these MMAs have read it
+                }
+                if (ok) tc::umma_commit(&done[piece & 1]);
+                g += len;
+            }
+            if (!ok) *failed = 1;
+        }
+        __syncwarp();
     } else {
-        if (tid == 0) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
-        // copies still on their way into this block's shared memory must land before it leaves:
-        // the most recent request of every stage is waited for (bounded)
-        if (tid == 32)
-            for (int32_t q = max(issued - SH_STAGES, 0); q < issued; ++q)
-                tc::mbar_wait(&full[q % SH_STAGES], (uint32_t)(q / SH_STAGES) & 1u);
+        // ---- four warps move each finished piece from tensor memory to its slab (thread = row) --
+        const int32_t m = warp * 32 + lane;
+        int32_t piece = 0;
+        for (int64_t g = g0; g < g1; ++piece) {
+            const int32_t t = (int32_t)(g / sp.nkb), kb = (int32_t)(g % sp.nkb);
+            const int32_t len = (int32_t)min((int64_t)(sp.nkb - kb), g1 - g);
+            const LongTile lt = long_tile(P, t);
+            const int32_t slab = (int32_t)blockIdx.x - first_block_of(sp, t);
+            const uint32_t bad =
+                (*failed != 0 || !lt.ok || !tc::mbar_wait(&done[piece & 1], (uint32_t)(piece / 2) & 1u)) ? 1u : 0u;
+            uint32_t any_bad;
+            asm volatile(
+                "{\n\t.reg .pred p, q;\n\t"
+                "setp.ne.u32 p, %1, 0;\n\t"
+                "bar.red.or.pred q, 1, 128, p;\n\t"
+                "selp.u32 %0, 1, 0, q;\n\t}"
+                : "=r"(any_bad)
+                : "r"(bad)
+                : "memory");
+            if (any_bad) { *failed = 1; break; }
+            tc::tc_fence_after();
+            float *dst = P.ws + ((int64_t)slab * P.T + lt.row0 + m) * P.RS;
+#pragma unroll
+            for (int c = 0; c < RP; c += 16) {
+                uint32_t r[16];
+                tc::tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(piece & 1) * ACC + c, r);
+                tc::tmem_ld_wait();
+                if (m < lt.rows) {  // rows past a short tile's end belong to other tiles
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4)
+                        *reinterpret_cast<uint4 *>(dst + c + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+                }
+            }
+            tc::tc_fence_before();
+            tc::mbar_arrive(&acc_free[piece & 1]);
+            g += len;
+        }
     }
     tc::tc_fence_before();
     __syncthreads();
-    if (warp == 0) tc::tmem_dealloc(tmem, TMEM_COLS);
+    if (tid == 0 && *failed) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
+    if (warp == 4) tc::tmem_dealloc(tmem, TMEM_COLS);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -390,8 +464,8 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
     unsigned char *Vl = Vh + C::V_BYTES;
     uint64_t *full = reinterpret_cast<uint64_t *>(Vl + C::V_BYTES);
     uint64_t *mma_done = full + S;
-    uint64_t *freed = mma_done + S;     // the epilogue is done with a stage and its store has read it
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(freed + S);
+    uint64_t *epi_done = mma_done + S;  // every epilogue thread has finished its row of the stage
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(epi_done + S);
     volatile int32_t *failed = reinterpret_cast<volatile int32_t *>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -408,7 +482,7 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
         for (int s = 0; s < S; ++s) {
             tc::mbar_init(&full[s], 1);
             tc::mbar_init(&mma_done[s], 1);
-            tc::mbar_init(&freed[s], 1);
+            tc::mbar_init(&epi_done[s], TC_ROWS);
         }
         *failed = 0;
         tc::fence_mbar_init();
@@ -417,9 +491,11 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
         tc::tmem_alloc(tmem_slot, C::TMEM_COLS);
         tc::tmem_relinquish();
     }
-    // v = sum of the K-slice partials (in order); thread = row.  Stored as bf16 high and low parts
+    // v = sum of the tile's pieces (in order); thread = row.  Stored as bf16 high and low parts
     // in the no-swizzle K-major layout: 8 x 8 core matrices of 128 bytes, the core matrix of row
     // group mg and rank group kg at (kg * 16 + mg) * 128 bytes.
+    const ShrinkSplit sp = shrink_split(P.list[0], P.tv.d_in, P.KS, P.shrink_grid);
+    const int32_t n_pieces = last_block_of(sp, (int32_t)blockIdx.x) - first_block_of(sp, (int32_t)blockIdx.x) + 1;
     if (tid < TC_ROWS) {
         const int32_t m = tid;
         const float *src = P.ws + ((int64_t)lt.row0 + m) * P.RS;
@@ -429,7 +505,7 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
             float v[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) v[e] = 0.0f;
-            for (int32_t q = 0; q < P.KS && m < lt.rows; ++q) {   // rows past a short tile's end stay zero
+            for (int32_t q = 0; q < n_pieces && m < lt.rows; ++q) {   // rows past a short tile's end stay zero
                 const float4 a = *reinterpret_cast<const float4 *>(src + q * ks_stride + kg * 8);
                 const float4 b = *reinterpret_cast<const float4 *>(src + q * ks_stride + kg * 8 + 4);
                 v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
@@ -483,24 +559,37 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
     };
 
     if (warp == 4) {
-        // ---- producer: one thread requests tiles S - 2 blocks ahead and issues each block's MMAs
-        // as soon as its tiles have landed; it never waits for an epilogue that is under way ------
+        // ---- one thread issues each block's MMAs as soon as its tiles have landed; it only ever
+        // waits for data --------------------------------------------------------------------------
+        if (lane == 0) {
+            for (int32_t j = 0; j < nblk; ++j) {
+                if (*failed || !issue_mma(j)) { *failed = 1; break; }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 5) {
+        // ---- one thread owns the stages' life cycle: it requests the first S blocks, and whenever
+        // the epilogue has finished a block it sends the tile out (TMA store), waits until the
+        // store has read the stage and requests the block that reuses it.  Every stage that is not
+        // being finished or stored therefore has a load in flight. ---------------------------------
         if (lane == 0) {
             int32_t issued = 0;
-            for (int32_t j = 0; j < nblk && j < S - 2; ++j, ++issued) issue_load(j);
-            for (int32_t j = 0; j < nblk && ok; ++j) {
-                if (*failed) break;
-                ok = issue_mma(j);
-                const int32_t n = j + S - 2;          // next block to request
-                if (ok && n < nblk) {
-                    if (n >= S) ok = tc::mbar_wait(&freed[n % S], (uint32_t)(n / S - 1) & 1u);
-                    if (ok) {
-                        issue_load(n);
-                        ++issued;
-                    }
+            for (int32_t j = 0; j < nblk && j < S; ++j, ++issued) issue_load(j);
+            for (int32_t j = 0; j < nblk; ++j) {
+                const int s = j % S;
+                if (!tc::mbar_wait(&epi_done[s], (uint32_t)(j / S) & 1u) || *failed) { ok = false; break; }
+                if (lt.rows == TC_ROWS) {
+                    tc::tma_store_2d(&map_y, (b0 + j) * 64, lt.t0, stages + s * C::STAGE);
+                    tc::bulk_commit();
+                    tc::bulk_wait_read<0>();
+                }
+                if (j + S < nblk) {
+                    issue_load(j + S);
+                    ++issued;
                 }
             }
-            if (!ok || *failed) {
+            tc::bulk_wait_read<0>();
+            if (!ok) {
                 *failed = 1;
                 // copies still on their way into this block's shared memory must land before it
                 // leaves: the most recent request of every stage is waited for (bounded)
@@ -556,22 +645,11 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
                             *reinterpret_cast<uint4 *>(yrow + chunk * 8) =
                                 *reinterpret_cast<const uint4 *>(tile + m * 128 + ((chunk ^ (m & 7)) << 4));
                 }
-                asm volatile("bar.sync 1, 128;" ::: "memory");   // every row has left the stage
-                if (tid == 0) tc::mbar_arrive(&freed[s]);
             } else {
                 tc::fence_proxy_async();    // the tile is read by the TMA store
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (tid == 0) {
-                    tc::tma_store_2d(&map_y, (b0 + j) * 64, lt.t0, tile);
-                    tc::bulk_commit();
-                    if (j > 0) {
-                        tc::bulk_wait_read<1>();      // the store before this one has read its stage
-                        tc::mbar_arrive(&freed[(j - 1) % S]);
-                    }
-                }
             }
+            tc::mbar_arrive(&epi_done[s]);  // 128 arrivals: every row of the stage is finished
         }
-        if (tid == 0) tc::bulk_wait_read<0>();
     }
     if (tid == 0 && *failed) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
     tc::tc_fence_before();
@@ -610,7 +688,7 @@ static bool make_map_2d(CUtensorMap *m, const void *base, int64_t rows, int64_t 
     cuuint32_t box[2] = {64, (cuuint32_t)TC_ROWS};
     cuuint32_t estr[2] = {1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 // 3-D view of one target's matrices in the pool: [slot][r_max rows][d columns]; box = 64 x box_rows x 1
@@ -623,7 +701,7 @@ static bool make_map_3d(CUtensorMap *m, const void *base, int64_t d, int64_t r_m
     cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -647,7 +725,7 @@ static lora_status_t launch_tc_bucket(lora_pool_t *pool, const TcParams &P, cons
                                            ExpandCfg<RP>::SMEM));
         attr_done = true;
     }
-    tc_shrink_kernel<RP><<<dim3(units, P.KS), TC_THREADS, SH_SMEM, stream>>>(P, mx, ma);
+    tc_shrink_kernel<RP><<<P.shrink_grid, TCS_THREADS, SH_SMEM, stream>>>(P, mx, ma);
     lora_status_t s = count_launch();
     if (s != LORA_OK) return s;
     tc_expand_kernel<RP><<<dim3(units, P.NS), TCX_THREADS, ExpandCfg<RP>::SMEM, stream>>>(P, mb, myb, my);
@@ -656,9 +734,10 @@ static lora_status_t launch_tc_bucket(lora_pool_t *pool, const TcParams &P, cons
 
 // Runs the long tiles of a batch.  Returns LORA_OK with *handled = false when the path does not
 // apply (no tensor-map support, misaligned operands); the caller then gives every tile to the
-// fused kernel.
+// fused kernel.  check_only: decide, launch nothing.
 lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, void *workspace,
-                                   size_t workspace_bytes, cudaStream_t stream, bool *handled) {
+                                   size_t workspace_bytes, cudaStream_t stream, bool *handled,
+                                   bool check_only) {
     *handled = false;
     if (!AP.meta || AP.tile_m != TC_ROWS || AP.T < TC_ROWS) return LORA_OK;
     // Short batches stay on the stream kernel alone (tuning key 4 = 2 forces this path whenever it
@@ -673,16 +752,12 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
     const int32_t max_long = (AP.T + TC_MIN_ROWS - 1) / TC_MIN_ROWS < AP.T / TC_ROWS + AP.meta_slots
                                  ? (AP.T + TC_MIN_ROWS - 1) / TC_MIN_ROWS
                                  : AP.T / TC_ROWS + AP.meta_slots;   // bound on tiles this path takes
-    int32_t KS = next_pow2((2 * pool->sm_count + max_long - 1) / max_long);
-    if (KS > 8) KS = 8;
-    const int32_t nkb = (AP.tv.d_in + 63) / 64;
-    while (KS > 1 && KS > nkb) KS >>= 1;
     const size_t per_split = (size_t)AP.T * RS * sizeof(float);
     // the work list (count + tile numbers) sits at the end of the workspace
     const size_t list_bytes = (((size_t)max_long + 1) * sizeof(int32_t) + 15) & ~(size_t)15;
     if (!workspace || workspace_bytes < list_bytes + per_split || ((uintptr_t)workspace & 15)) return LORA_OK;
     const size_t ws_partials = (workspace_bytes - list_bytes) & ~(size_t)15;
-    while (KS > 1 && per_split * KS > ws_partials) KS >>= 1;
+    int32_t KS = (int32_t)(ws_partials / per_split < 8 ? ws_partials / per_split : 8);   // slabs of partials
     int32_t NS = (4 * pool->sm_count + max_long - 1) / max_long;
     const int32_t nblk = (AP.tv.d_out + 63) / 64;
     if (NS > nblk) NS = nblk;
@@ -704,6 +779,11 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
     P.target_rows = pool->r_max;
     P.list = reinterpret_cast<int32_t *>((char *)workspace + ws_partials);
     P.list_cap = max_long;
+    P.shrink_grid = 2 * pool->sm_count;   // two blocks fit on an SM: the grid fills the GPU exactly once
+    if (check_only) {   // nothing has been launched: the caller only asks whether the path applies
+        *handled = true;
+        return LORA_OK;
+    }
     const int32_t units = max_long;   // block columns: one per work-list entry, the unused ones leave at once
     tc_worklist_kernel<<<1, 256, 0, stream>>>(P);
     {

@@ -141,6 +141,9 @@ struct lora_pool {
     // Tensor maps of the fused kernel in the pool's device buffer, written at creation: per
     // target 8 for A and 8 for B (one per number of rank rows 8, 16, .. 64 a tile load fetches).
     CUtensorMap *maps_dev = nullptr;
+    // lora_sgmv_apply runs the tiles its tensor-core kernels leave over beside those kernels
+    cudaStream_t side_stream = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     // What the fused kernel's launcher has set or asked for this pool's device (dynamic
     // shared-memory limit, resident clusters), per kernel variant; part of the handle, so pools
     // used from different threads share nothing.

@@ -163,7 +163,7 @@ __device__ __forceinline__ void producer(const FusedParams &P, unsigned char *sm
     uint32_t ph = 0;
     bool ok = true, have_pend = false, waited = !P.early;
     PUnit pend;
-    int32_t pend_rowid = 0, pend_entry = 0;
+    int32_t pend_rowid = 0, pend_entry = 0, n_run = 0;
     bool sent_final = false;
     for (int32_t i = 0;; ++i) {
         const bool real = g < total;
@@ -176,7 +176,12 @@ __device__ __forceinline__ void producer(const FusedParams &P, unsigned char *sm
         fetch(un_, next_real, rec_n, rowid_n);   // the next unit's record, meanwhile
         PUnit un = p_decode(P, crank, bcast(rec), item);
         if (!real) un.run = false;   // past the end: only the last unit's expand jobs are left
-        const int32_t entry = i & (UNIT_ENTRIES - 1);
+        // Entries are numbered by the units that run, not by the units walked: a cluster that
+        // skips units between two that run must not come back to an entry still in use (the
+        // entry of a unit is read until its last expand chunk, which follows the next running
+        // unit's shrink chunks in the ring).
+        const int32_t entry = n_run & (UNIT_ENTRIES - 1);
+        if (un.run) ++n_run;
         if (un.run) {
             // the unit's entry; made visible to the consumers by the arrival on the barrier of
             // the unit's first job

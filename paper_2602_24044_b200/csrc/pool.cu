@@ -112,6 +112,15 @@ lora_status_t lora_pool_bytes(const lora_pool_desc_t *desc, size_t *bytes) {
     return LORA_OK;
 }
 
+static void release_sync_objects(lora_pool_t *p) {
+    if (p->fence) cudaEventDestroy(p->fence);
+    if (p->ev_fork) cudaEventDestroy(p->ev_fork);
+    if (p->ev_join) cudaEventDestroy(p->ev_join);
+    if (p->side_stream) cudaStreamDestroy(p->side_stream);
+    p->fence = p->ev_fork = p->ev_join = nullptr;
+    p->side_stream = nullptr;
+}
+
 lora_status_t lora_pool_create(const lora_pool_desc_t *desc, lora_pool_t **out) {
     if (!out) return LORA_ERR_INVALID_ARG;
     *out = nullptr;
@@ -154,16 +163,19 @@ lora_status_t lora_pool_create(const lora_pool_desc_t *desc, lora_pool_t **out) 
     p->table_host.assign(p->num_slots, empty);
     p->ready.assign(p->num_slots, nullptr);
     cudaError_t e = cudaEventCreateWithFlags(&p->fence, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->side_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaMemset(p->base, 0, L.off_staging);   // status, table, tensor maps
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount,
                                                      desc->device);
     if (e != cudaSuccess) {
-        if (p->fence) cudaEventDestroy(p->fence);
+        release_sync_objects(p);
         delete p;
         return cuda_fail(e);
     }
     if ((s = build_fused_maps(p)) != LORA_OK) {
-        cudaEventDestroy(p->fence);
+        release_sync_objects(p);
         delete p;
         return s;
     }
@@ -176,7 +188,7 @@ lora_status_t lora_pool_destroy(lora_pool_t *pool) {
     DeviceGuard guard(pool->device);
     for (cudaEvent_t ev : pool->ready)
         if (ev) cudaEventDestroy(ev);
-    if (pool->fence) cudaEventDestroy(pool->fence);
+    release_sync_objects(pool);
     delete pool;
     return LORA_OK;
 }

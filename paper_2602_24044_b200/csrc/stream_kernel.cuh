@@ -185,7 +185,7 @@ __device__ __forceinline__ void producer(const FusedParams &P, unsigned char *sm
     uint32_t ph = 0;
     bool ok = true, have_pend = false, waited = !P.early, sent_final = false;
     PUnit pend;
-    int32_t pend_rowid = 0, pend_entry = 0;
+    int32_t pend_rowid = 0, pend_entry = 0, n_run = 0;
     // waits until stage st may be refilled; false once a wait has run out
     auto stage_free = [&]() {
         if (q >= S && ok) {
@@ -213,7 +213,12 @@ __device__ __forceinline__ void producer(const FusedParams &P, unsigned char *sm
         // per-token mode: a slot id that is neither -1 nor an occupied slot is counted once
         if (real && !P.meta && rb.x == -1 && rb.y && crank == 0 && un.item == 0 && lane == 0)
             atomicAdd(&P.pool.status[STATUS_INVALID_TOKENS], 1);
-        const int32_t entry = i & (UNIT_ENTRIES - 1);
+        // Entries are numbered by the units that run, not by the units walked: a cluster that
+        // skips units between two that run must not come back to an entry still in use (the
+        // entry of a unit is read until its last expand chunk, which follows the next running
+        // unit's shrink chunks in the ring).
+        const int32_t entry = n_run & (UNIT_ENTRIES - 1);
+        if (un.run) ++n_run;
         if (un.run) {
             // the unit's entry; made visible to the consumers by the arrival on the barrier of
             // the unit's first job

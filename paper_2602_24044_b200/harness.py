@@ -155,6 +155,10 @@ class Session:
         sidx = self.slot_idx_dev if slot_idx_dev is None else slot_idx_dev
         y = y_base if in_place else torch.empty_like(y_base)
         with torch.cuda.stream(self.compute):
+            if not in_place:
+                # a row the kernels never write must not pass for a result left over in recycled
+                # memory: the output starts as a huge finite value in every element
+                y.view(torch.int16).fill_(0x7F7F)
             meta = None
             if grouped or kind == "sgmv":
                 if rebuild or self.meta_shape is None:
