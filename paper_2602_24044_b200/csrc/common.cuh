@@ -155,6 +155,7 @@ struct lora_pool {
     bool twophase_attr_done = false;
     bool tc_attr_done[3] = {false, false, false};   // rank buckets 16, 32, 64
     size_t seg_attr_smem = 0, seg_attr_chunked = 0;
+    size_t seg_attr_chunked_wide = 0;
 
     // Shapes of the metadata tables built through this handle (the table itself lives on the
     // device; apply calls need T and tile_m on the host to size their grids).

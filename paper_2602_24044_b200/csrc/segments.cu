@@ -231,10 +231,15 @@ build_segments_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int
 // (counts, prefix sums, first and last token of every tile); the writes to global memory are
 // divided: a block writes the perm entries of its own chunks and the records of its own slots.
 // Tokens without an occupied slot are counted in an extra column and land behind the active ones.
-__global__ void __launch_bounds__(SEG_THREADS)
+// The two passes over the token list are chains of shared-memory updates per warp, so their length
+// is the number of chunks a warp owns: 32 warps for the longest batches, 8 below that (where the
+// larger block only costs more at its barriers).
+template <int SEGC_THREADS>
+__global__ void __launch_bounds__(SEGC_THREADS)
 build_segments_chunked_kernel(PoolView pool, const int32_t *__restrict__ slot_idx_g, int32_t T,
                               int32_t tile_m, int32_t long_min, int32_t *meta, int32_t CH, int32_t C) {
     extern __shared__ int32_t sm[];
+    constexpr int SEGC_WARPS = SEGC_THREADS / 32;
     const int32_t N = pool.num_slots, N1 = N + 1;
     const MetaLayout L = meta_layout(T, N, tile_m);
     int32_t *cnt = sm;             // [N] tokens per slot
@@ -247,7 +252,7 @@ build_segments_chunked_kernel(PoolView pool, const int32_t *__restrict__ slot_id
     int32_t *cnt2 = tok + T;       // [C][N + 1] per chunk and slot: count, then running position
     int32_t *tfirst = cnt2 + (int64_t)C * N1;   // [cap_tile] first token id of a tile
     int32_t *tlast = tfirst + L.cap_tile;       // [cap_tile] last token id of a tile
-    __shared__ int32_t warp_tot[4][SEG_WARPS];
+    __shared__ int32_t warp_tot[4][SEGC_WARPS];
     __shared__ int32_t totals[4];
     __shared__ int32_t n_invalid_s;
 
@@ -255,12 +260,12 @@ build_segments_chunked_kernel(PoolView pool, const int32_t *__restrict__ slot_id
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    for (int32_t s = tid; s < N; s += SEG_THREADS) {
+    for (int32_t s = tid; s < N; s += SEGC_THREADS) {
         cnt[s] = 0;
         occ[s] = pool.table[s].loaded;
     }
-    for (int32_t i = tid; i < C * N1; i += SEG_THREADS) cnt2[i] = 0;
-    for (int32_t t = tid; t < T; t += SEG_THREADS) tok[t] = slot_idx_g[t];
+    for (int32_t i = tid; i < C * N1; i += SEGC_THREADS) cnt2[i] = 0;
+    for (int32_t t = tid; t < T; t += SEGC_THREADS) tok[t] = slot_idx_g[t];
     if (tid == 0) n_invalid_s = 0;
     __syncthreads();
 
@@ -273,7 +278,7 @@ build_segments_chunked_kernel(PoolView pool, const int32_t *__restrict__ slot_id
     };
 
     // ---- 1. counts per chunk and column --------------------------------------------------------
-    for (int32_t c = warp; c < C; c += SEG_WARPS) {
+    for (int32_t c = warp; c < C; c += SEGC_WARPS) {
         const int32_t t0 = c * CH, t1 = min(T, t0 + CH);
         for (int32_t base = t0; base < t1; base += 32) {
             int32_t s; bool valid, act;
@@ -287,7 +292,7 @@ build_segments_chunked_kernel(PoolView pool, const int32_t *__restrict__ slot_id
     }
     __syncthreads();
     // ---- 2. per column: exclusive prefix over the chunks; per slot: totals and prefix sums -------
-    for (int32_t col = tid; col < N1; col += SEG_THREADS) {
+    for (int32_t col = tid; col < N1; col += SEGC_THREADS) {
         int32_t run = 0;
         for (int32_t c = 0; c < C; ++c) {
             const int32_t v = cnt2[c * N1 + col];
@@ -297,7 +302,7 @@ build_segments_chunked_kernel(PoolView pool, const int32_t *__restrict__ slot_id
         if (col < N) cnt[col] = run;
     }
     __syncthreads();
-    const int32_t per = (N + SEG_THREADS - 1) / SEG_THREADS;
+    const int32_t per = (N + SEGC_THREADS - 1) / SEGC_THREADS;
     const int32_t lo = min(tid * per, N), hi = min(lo + per, N);
     const int32_t ppt = (tile_m + 15) / 16;
     auto pieces_of = [&](int32_t n) { return (n / tile_m) * ppt + ((n % tile_m) + 15) / 16; };
@@ -336,13 +341,13 @@ build_segments_chunked_kernel(PoolView pool, const int32_t *__restrict__ slot_id
         rt += (cnt[s] + tile_m - 1) / tile_m;
         rp += pieces_of(cnt[s]);
     }
-    if (tid == SEG_THREADS - 1) { totals[0] = rc; totals[1] = rz; totals[2] = rt; totals[3] = rp; }
+    if (tid == SEGC_THREADS - 1) { totals[0] = rc; totals[1] = rz; totals[2] = rt; totals[3] = rp; }
     __syncthreads();
     const int32_t n_active = totals[0], n_seg = totals[1], n_tile = totals[2], n_piece = totals[3];
 
     // ---- 3. position of every token; first and last token of every tile --------------------------
     int32_t *perm = meta + L.perm;
-    for (int32_t c = warp; c < C; c += SEG_WARPS) {
+    for (int32_t c = warp; c < C; c += SEGC_WARPS) {
         const int32_t t0 = c * CH, t1 = min(T, t0 + CH);
         const bool mine = (c % (int32_t)gridDim.x) == (int32_t)blockIdx.x;
         for (int32_t base = t0; base < t1; base += 32) {
@@ -371,7 +376,7 @@ build_segments_chunked_kernel(PoolView pool, const int32_t *__restrict__ slot_id
     __syncthreads();
 
     // ---- 4. segment, tile and unit records of this block's slots ---------------------------------
-    for (int32_t s = blockIdx.x * SEG_WARPS + warp; s < N; s += gridDim.x * SEG_WARPS) {
+    for (int32_t s = blockIdx.x * SEGC_WARPS + warp; s < N; s += gridDim.x * SEGC_WARPS) {
         const int32_t n = cnt[s];
         if (n == 0) continue;
         const int32_t p0 = start[s], seg = segid[s];
@@ -422,13 +427,13 @@ build_segments_chunked_kernel(PoolView pool, const int32_t *__restrict__ slot_id
         meta[L.seg_start + n_seg] = n_active;
         if (n_invalid) atomicAdd(&pool.status[STATUS_INVALID_TOKENS], n_invalid);
     }
-    for (int32_t i = n_seg + tid; i < L.cap_seg; i += SEG_THREADS) {
+    for (int32_t i = n_seg + tid; i < L.cap_seg; i += SEGC_THREADS) {
         meta[L.seg_slot + i] = -1;
         meta[L.seg_rank + i] = -1;
         meta[L.seg_flags + i] = -1;
     }
-    for (int32_t i = n_seg + 1 + tid; i <= L.cap_seg; i += SEG_THREADS) meta[L.seg_start + i] = -1;
-    for (int32_t i = n_tile + tid; i < L.cap_tile; i += SEG_THREADS) {
+    for (int32_t i = n_seg + 1 + tid; i <= L.cap_seg; i += SEGC_THREADS) meta[L.seg_start + i] = -1;
+    for (int32_t i = n_tile + tid; i < L.cap_tile; i += SEGC_THREADS) {
         meta[L.tile_seg + i] = -1;
         meta[L.tile_row0 + i] = -1;
         meta[L.tile_rows + i] = -1;
@@ -450,19 +455,28 @@ lora_status_t launch_build_segments(lora_pool_t *pool, const int32_t *slot_idx_d
         const size_t words = 6 * (size_t)N + (size_t)T + (size_t)C * (N + 1) + 2 * (size_t)L.cap_tile;
         if (words * sizeof(int32_t) <= 200 * 1024) {
             const size_t smem = words * sizeof(int32_t);
-            size_t &attr_chunked = pool->seg_attr_chunked;
+            const bool wide = T >= 8192;
+            size_t &attr_chunked = wide ? pool->seg_attr_chunked_wide : pool->seg_attr_chunked;
             if (attr_chunked == 0) attr_chunked = 48 * 1024;
             if (smem > attr_chunked) {
-                cudaError_t e = cudaFuncSetAttribute(build_segments_chunked_kernel,
-                                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                cudaError_t e = wide ? cudaFuncSetAttribute(build_segments_chunked_kernel<1024>,
+                                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                                     : cudaFuncSetAttribute(build_segments_chunked_kernel<256>,
+                                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
                 if (e != cudaSuccess) return cuda_fail(e);
                 attr_chunked = smem;
             }
-            int grid = (N + SEG_WARPS - 1) / SEG_WARPS;
-            if (grid < (C + SEG_WARPS - 1) / SEG_WARPS) grid = (C + SEG_WARPS - 1) / SEG_WARPS;
+            // every block builds the tables; the blocks share the writes (chunks of perm, slots)
+            const int warps = wide ? 32 : 8;
+            int grid = (N + warps - 1) / warps;
+            if (grid < (C + 7) / 8) grid = (C + 7) / 8;
             if (grid > pool->sm_count) grid = pool->sm_count;
-            build_segments_chunked_kernel<<<grid, SEG_THREADS, smem, stream>>>(
-                pool->view(), slot_idx_dev, T, tile_m, long_min, (int32_t *)meta_dev, CH, C);
+            if (wide)
+                build_segments_chunked_kernel<1024><<<grid, 1024, smem, stream>>>(
+                    pool->view(), slot_idx_dev, T, tile_m, long_min, (int32_t *)meta_dev, CH, C);
+            else
+                build_segments_chunked_kernel<256><<<grid, 256, smem, stream>>>(
+                    pool->view(), slot_idx_dev, T, tile_m, long_min, (int32_t *)meta_dev, CH, C);
             return count_launch();
         }
     }
