@@ -158,7 +158,7 @@ __host__ __device__ constexpr uint32_t instr_desc(uint32_t M, uint32_t N, uint32
 
 constexpr int TCX_THREADS = 192;   // expand: four epilogue warps, one warp that issues MMAs, one that issues copies
 constexpr int TC_ROWS = 128;       // rows of a long tile
-constexpr int SH_STAGES = 4;       // shrink: ring of (x tile, A tile) stages
+constexpr int SH_STAGES = 3;       // shrink: ring of (x tile, A tile) stages
 constexpr int XT_BYTES = TC_ROWS * 128;   // 128 rows x 64 bf16
 
 struct TcParams {
@@ -440,7 +440,7 @@ struct ExpandCfg {
 #ifdef LORA_TC_EXPAND_STAGES
     static constexpr int STAGES = LORA_TC_EXPAND_STAGES;
 #else
-    static constexpr int STAGES = 4;   // 2 blocks per SM up to rank 32; deeper rings measured slower
+    static constexpr int STAGES = 3;   // three stages leave room for a block of the fused kernel beside two of these
 #endif
     static constexpr int BT_BYTES = RP * 128;                       // RP rank rows x 64 columns
     static constexpr int STAGE = XT_BYTES + ((BT_BYTES + 1023) & ~1023);   // y_base/out tile + B tile
@@ -759,6 +759,7 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
     const size_t ws_partials = (workspace_bytes - list_bytes) & ~(size_t)15;
     int32_t KS = (int32_t)(ws_partials / per_split < 8 ? ws_partials / per_split : 8);   // slabs of partials
     int32_t NS = (4 * pool->sm_count + max_long - 1) / max_long;
+    if (pool->tuning[8] > 0) NS = pool->tuning[8];   // tuning key 8: column splits of a tile in the expand
     const int32_t nblk = (AP.tv.d_out + 63) / 64;
     if (NS > nblk) NS = nblk;
     if (NS < 1) NS = 1;
