@@ -141,9 +141,11 @@ class Session:
     def apply(self, call: int = 0, x: Optional[torch.Tensor] = None,
               y_base: Optional[torch.Tensor] = None, *, kind: Optional[str] = None,
               grouped: bool = True, in_place: bool = False,
-              slot_idx_dev: Optional[torch.Tensor] = None, rebuild: bool = True) -> torch.Tensor:
+              slot_idx_dev: Optional[torch.Tensor] = None, rebuild: bool = True,
+              ws_bytes: Optional[int] = None) -> torch.Tensor:
         """One apply on the compute stream; returns y (device tensor).  x / y_base default to
-        the workload's activations for `call`."""
+        the workload's activations for `call`.  ws_bytes: how much of the workspace the call is
+        told about (default: all of it)."""
         wl = self.wl
         target = wl.calls[call]
         d_in, d_out = wl.targets[target]
@@ -170,7 +172,7 @@ class Session:
                               y.stride(0), sidx, T, meta, self.ws, stream=self.compute)
             else:
                 lb.sgmv_apply(self.pool, tp, x, x.stride(0), y_base, y_base.stride(0), y,
-                              y.stride(0), meta, T, self.ws, stream=self.compute)
+                              y.stride(0), meta, T, self.ws, ws_bytes, stream=self.compute)
         return y
 
     def close(self):

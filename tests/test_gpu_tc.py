@@ -68,3 +68,58 @@ def test_mixed_batch_scattered_and_long_tiles():
     y_ref, _ = oracle_full(wl)
     y, _ = _run(wl)
     check_tolerance(y, y_ref, what="mixed batch")
+
+
+@pytest.mark.parametrize("slabs", [1, 2, 3, 5, 8])
+def test_workspace_that_holds_few_partial_slabs(slabs):
+    """The shrink cuts every tile's K range into pieces, one fp32 slab of the workspace per piece;
+    a smaller workspace means fewer, longer pieces (one slab: whole tiles only).  Same result."""
+    wl = W.make_custom(1000, 1024, 1536, 5, [8, 16, 32], kind="sgmv", index="sorted", tile_m=128,
+                       scale=[0.6, 1.3], weight_mode="unitB", seed=56)
+    y_ref, _ = oracle_full(wl)
+    per_slab = wl.T * 32 * 4            # tokens x rank bucket of the pool x fp32
+    y, n = _run(wl, ws_bytes=slabs * per_slab + 4096)   # the work list fits in the slack
+    check_tolerance(y, y_ref, what="%d slabs" % slabs)
+    _, n_fused = _run(wl, tuning={4: 1})
+    assert n > n_fused                  # the tensor-core kernels took their tiles
+
+
+def test_prefill_apply_in_a_cuda_graph():
+    """lora_sgmv_apply forks the leftover tiles onto the pool's own stream and joins it back; the
+    whole call must be capturable and a replay must reproduce the eager result bit for bit."""
+    import torch
+    from paper_2602_24044_b200 import binding as lb
+    from paper_2602_24044_b200.harness import Session, bf16_bits, bf16_tensor
+    rng = np.random.default_rng(57)
+    dec = rng.integers(0, 12, 90)
+    slot_idx = np.concatenate([np.repeat([2, 5], 300), dec, np.repeat([9], 200)]).astype(np.int32)
+    wl = W.make_custom(0, 1024, 768, 12, [8, 16, 32], kind="sgmv", tile_m=128, scale=0.9,
+                       weight_mode="unitB", slot_idx=slot_idx, seed=57)
+    y_ref, _ = oracle_full(wl)
+    with Session(wl, tuning={4: 2}) as s:
+        x_h, yb_h = wl.activations(0)
+        x, yb = bf16_tensor(x_h, s.device), bf16_tensor(yb_h, s.device)
+        y = torch.empty_like(yb)
+        nwords = lb.segments_bytes(wl.T, wl.num_slots, wl.tile_m) // 4
+        meta = torch.empty(nwords, dtype=torch.int32, device=s.device)
+
+        def step():
+            lb.build_segments(s.pool, s.slot_idx_dev, wl.T, wl.tile_m, wl.long_min, meta, stream=s.compute)
+            lb.sgmv_apply(s.pool, 0, x, x.shape[1], yb, yb.shape[1], y, y.shape[1], meta, wl.T, s.ws,
+                          stream=s.compute)
+
+        with torch.cuda.stream(s.compute):
+            step()
+        eager = bf16_bits(y).copy()
+        check_tolerance(eager, y_ref, what="eager")
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s.compute):
+            step()
+            step()
+        for _ in range(3):
+            y.view(torch.int16).fill_(0x7F7F)
+            torch.cuda.synchronize()
+            with torch.cuda.stream(s.compute):
+                g.replay()
+            assert np.array_equal(bf16_bits(y), eager)
+        assert s.status()[1] == 0
