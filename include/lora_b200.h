@@ -173,7 +173,8 @@ lora_status_t lora_pool_selftest_wait_expiry(lora_pool_t *pool, int32_t polls, i
  *   key 1  fused kernel: blocks per cluster (1, 2, 4, 8)
  *   key 2  programmatic dependent launch of the fused kernel: 2 = never
  *   key 3  fused kernel: upper bound on the clusters in the grid
- *   key 4  tensor-core kernels of lora_sgmv_apply: 1 = never, 2 = whenever they apply
+ *   key 4  tensor-core kernels of lora_sgmv_apply: 1 = never, 2 = whenever they apply (read by
+ *          lora_build_segments, which writes their tile list, and by the apply)
  *   key 5  fused kernel: stages of the shared-memory ring (2 .. 4)
  *   key 6  lora_sgmv_apply: 1 = the tiles the tensor-core kernels leave over run after them on the
  *          caller's stream, not beside them on the pool's own stream
@@ -257,8 +258,9 @@ lora_status_t lora_pool_plan(size_t bytes_budget, const lora_target_t *targets, 
  *                each segment cut into pieces of at most tile_m rows (positions in perm)
  *   (then words private to the library: one flag word per tile, and from the next 16-byte
  *    boundary a 4-word record per
- *    tile, and a 4-word record plus 16 row ids per piece of at most 16 rows of a tile;
- *    lora_segments_bytes counts them)
+ *    tile, a 4-word record plus 16 row ids per piece of at most 16 rows of a tile, and the
+ *    list of the tiles lora_sgmv_apply gives to its tensor-core kernels (written by a second
+ *    small launch when the batch qualifies for them); lora_segments_bytes counts them)
  * Unused entries are -1.  A token is active iff its slot id names an occupied slot; a token
  * that is neither active nor -1 is invalid (counted in header and in the pool's status word 0).
  * The result is an exact integer function of its inputs.
@@ -278,9 +280,8 @@ lora_status_t lora_build_segments(lora_pool_t *pool, const int32_t *slot_idx_dev
  * not overlapping it.  Tokens without an active slot get y = y_base bit for bit.  Row t of y
  * depends only on row t of x and y_base, the token's slot and the pool.
  * workspace: dev scratch of >= lora_workspace_bytes(pool, T) bytes (fp32 partial products
- * v = x . A_i between the two phases of the tensor-core and two-phase kernels and the
- * tensor-core path's list of long tiles; the fused kernels keep v on chip), contents undefined
- * afterwards; calls sharing a workspace must be ordered on
+ * v = x . A_i between the two phases of the tensor-core and two-phase kernels; the fused
+ * kernels keep v on chip), contents undefined afterwards; calls sharing a workspace must be ordered on
  * one stream.
  * Ordering: every apply is ordered behind the lora_build_segments call that wrote its table.
  * Later applies on the same table may start reading the table and the pool (never x or y_base)

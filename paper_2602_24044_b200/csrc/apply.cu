@@ -117,7 +117,7 @@ extern "C" {
 lora_status_t lora_workspace_bytes(const lora_pool_t *pool, int32_t T_max, size_t *bytes) {
     if (!pool || !bytes) return LORA_ERR_INVALID_ARG;
     if (T_max < 0) return LORA_ERR_SHAPE;
-    // eight split-K partials of v, and the tensor-core path's list of long tiles behind them
+    // eight fp32 slabs for the partial v of the tensor-core shrink's pieces (and a little slack)
     const size_t T = (size_t)(T_max > 0 ? T_max : 1);
     *bytes = (size_t)8 * T * rank_bucket(pool->r_max) * sizeof(float) + ((T / 32 + 8) * sizeof(int32_t) + 15) / 16 * 16;
     return LORA_OK;

@@ -144,6 +144,11 @@ lora_status_t build_fused_maps(lora_pool_t *pool);
 lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, void *workspace,
                                    size_t workspace_bytes, cudaStream_t stream, bool *handled,
                                    bool check_only);
+// Whether a batch of T tokens built with tile_m would be given to the tensor-core kernels, and the
+// launch that writes their list of long tiles into the metadata (behind the build, same stream).
+bool tc_path_wanted(const lora_pool_t *pool, int32_t T, int32_t tile_m);
+lora_status_t launch_tc_worklist(lora_pool_t *pool, int32_t T, int32_t tile_m, void *meta_dev,
+                                 cudaStream_t stream);
 lora_status_t launch_build_segments(lora_pool_t *pool, const int32_t *slot_idx_dev, int32_t T,
                                     int32_t tile_m, int32_t long_min, void *meta_dev,
                                     cudaStream_t stream);

@@ -1,16 +1,19 @@
-// Tensor-core path of lora_sgmv_apply for LONG tiles: 128 consecutive tokens of one adapter
-// (prefill / chunked-prefill segments), y = y_base + s_i * (x . A_i) . B_i (paper Section 2.2).
+// Tensor-core path of lora_sgmv_apply for LONG tiles: runs of 32 .. 128 consecutive tokens of one
+// adapter (prefill / chunked-prefill segments), y = y_base + s_i * (x . A_i) . B_i (paper Section 2.2).
 //
 // Such a tile is a dense contraction, so it runs on the 5th-generation tensor cores:
-//   tc_shrink_kernel  V_part[128, r] = X[128, K-slice] . A_i[r, K-slice]^T
-//       X and A_i tiles arrive by TMA (128-byte swizzle) through a 4-stage mbarrier ring; one
-//       thread issues tcgen05.mma (M = 128, N = rank bucket, K = 16) with the accumulator in
-//       tensor memory; the partial of each K-slice goes to the fp32 workspace.
-//   tc_expand_kernel  Y[128, N-slice] = Y_base + s * V . B_i[r, N-slice]
-//       V = sum of the partials, carried as a high and a low bf16 part (two MMAs, ~16 mantissa
-//       bits); per 64-column block one TMA load of the B_i tile and of the y_base tile, MMA into a
-//       ring of tensor-memory accumulators, epilogue tcgen05.ld -> fused scale + residual add ->
-//       bf16 written in place into the y_base tile -> TMA store.
+//   tc_worklist_kernel  the long tiles of the batch, in tile order, as a compact list
+//   tc_shrink_kernel    V[128, r] = X[128, d_in] . A_i[r, d_in]^T, computed in pieces: the (tile,
+//       K-block) pairs of all tiles form one walk cut into equal spans, one per block of a grid
+//       that fills the GPU once.  X and A_i tiles arrive by TMA (128-byte swizzle) through a
+//       three-stage mbarrier ring; one thread requests them, one issues tcgen05.mma (M = 128,
+//       N = rank bucket, K = 16) with the accumulator in tensor memory, four warps write each
+//       finished piece to its fp32 slab of the workspace.
+//   tc_expand_kernel    Y[128, N-slice] = Y_base + s * V . B_i[r, N-slice]
+//       V = sum of the tile's pieces (in order), carried as a high and a low bf16 part (two MMAs,
+//       ~16 mantissa bits); per 64-column block one TMA load of the B_i tile and of the y_base
+//       tile, MMA into a ring of tensor-memory accumulators, epilogue tcgen05.ld -> fused scale +
+//       residual add -> bf16 written in place into the y_base tile -> TMA store.
 // Both kernels are HBM-bound streaming kernels: the tensor cores only keep the arithmetic off the
 // critical path.  Every wait on an mbarrier is bounded; on expiry the block records it in the
 // pool's status word, frees its tensor memory and leaves without storing.
@@ -19,6 +22,7 @@
 
 #include <cstdio>
 #include <cstdlib>
+#include <cstring>
 
 #include "apply_common.cuh"
 
@@ -172,7 +176,7 @@ struct TcParams {
     int32_t target_rows;    // r_max: rows of a slot's matrices
     __nv_bfloat16 *y;       // output, for tiles with fewer than 128 rows (stored row by row)
     int64_t ldy;
-    int32_t *list;          // work list in the workspace: [0] = number of long tiles, then their tile numbers
+    int32_t *list;          // list of long tiles in the metadata: [0] = their number, then their tile numbers
     int32_t list_cap;
 };
 
@@ -207,8 +211,9 @@ __device__ __forceinline__ LongTile long_tile(const TcParams &P, int32_t entry) 
 }
 
 // The tiles this path takes (runs of at least TC_MIN_ROWS consecutive tokens), in tile order, as a
-// compact list: the two kernels below then launch one block column per list entry instead of one
-// per tile of the batch (a mixed batch has hundreds of tiles and a handful of long ones).
+// compact list in the metadata buffer, written once behind the build (every apply on that table
+// reads it): the kernels below walk list entries, not the tiles of the batch (a mixed batch has
+// hundreds of tiles and a handful of long ones).
 __global__ void __launch_bounds__(256)
 tc_worklist_kernel(const TcParams P) {
     __shared__ int32_t warp_count[8];
@@ -732,6 +737,28 @@ static lora_status_t launch_tc_bucket(lora_pool_t *pool, const TcParams &P, cons
     return count_launch();
 }
 
+bool tc_path_wanted(const lora_pool_t *pool, int32_t T, int32_t tile_m) {
+    if (tile_m != TC_ROWS || T < TC_ROWS || pool->tuning[4] == 1 || pool->tuning[0] == 1) return false;
+    // Short batches stay on the stream kernel alone (tuning key 4 = 2: these kernels whenever they apply).
+    return T / TC_ROWS >= TC_MIN_TILES || pool->tuning[4] == 2;
+}
+
+lora_status_t launch_tc_worklist(lora_pool_t *pool, int32_t T, int32_t tile_m, void *meta_dev,
+                                 cudaStream_t stream) {
+    const MetaLayout L = meta_layout(T, pool->num_slots, tile_m);
+    if (L.words > 0x7fffffff) return LORA_ERR_SHAPE;
+    TcParams P;
+    memset(&P, 0, sizeof(P));
+    P.meta = (const int32_t *)meta_dev;
+    P.T = T;
+    P.moff_perm = (int32_t)L.perm;
+    P.moff_desc = (int32_t)L.tile_desc;
+    P.list = (int32_t *)meta_dev + L.long_list;
+    P.list_cap = L.cap_tile;
+    tc_worklist_kernel<<<1, 256, 0, stream>>>(P);
+    return count_launch();
+}
+
 // Runs the long tiles of a batch.  Returns LORA_OK with *handled = false when the path does not
 // apply (no tensor-map support, misaligned operands); the caller then gives every tile to the
 // fused kernel.  check_only: decide, launch nothing.
@@ -740,9 +767,7 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
                                    bool check_only) {
     *handled = false;
     if (!AP.meta || AP.tile_m != TC_ROWS || AP.T < TC_ROWS) return LORA_OK;
-    // Short batches stay on the stream kernel alone (tuning key 4 = 2 forces this path whenever it
-    // applies).
-    if (AP.T / TC_ROWS < TC_MIN_TILES && pool->tuning[4] != 2) return LORA_OK;
+    if (!tc_path_wanted(pool, AP.T, AP.tile_m)) return LORA_OK;
     if (!encode_fn()) return LORA_OK;
     // TMA wants 16-byte aligned bases and row pitches
     if ((((uintptr_t)AP.x | (uintptr_t)AP.yb | (uintptr_t)AP.y) & 15) || (AP.ldx % 8) || (AP.ldyb % 8) ||
@@ -752,12 +777,10 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
     const int32_t max_long = (AP.T + TC_MIN_ROWS - 1) / TC_MIN_ROWS < AP.T / TC_ROWS + AP.meta_slots
                                  ? (AP.T + TC_MIN_ROWS - 1) / TC_MIN_ROWS
                                  : AP.T / TC_ROWS + AP.meta_slots;   // bound on tiles this path takes
+    if (!pool->meta_has_list(AP.meta)) return LORA_OK;   // built before the batch qualified (tuning changed)
     const size_t per_split = (size_t)AP.T * RS * sizeof(float);
-    // the work list (count + tile numbers) sits at the end of the workspace
-    const size_t list_bytes = (((size_t)max_long + 1) * sizeof(int32_t) + 15) & ~(size_t)15;
-    if (!workspace || workspace_bytes < list_bytes + per_split || ((uintptr_t)workspace & 15)) return LORA_OK;
-    const size_t ws_partials = (workspace_bytes - list_bytes) & ~(size_t)15;
-    int32_t KS = (int32_t)(ws_partials / per_split < 8 ? ws_partials / per_split : 8);   // slabs of partials
+    if (!workspace || workspace_bytes < per_split || ((uintptr_t)workspace & 15)) return LORA_OK;
+    int32_t KS = (int32_t)(workspace_bytes / per_split < 8 ? workspace_bytes / per_split : 8);   // slabs of partials
     int32_t NS = (4 * pool->sm_count + max_long - 1) / max_long;
     if (pool->tuning[8] > 0) NS = pool->tuning[8];   // tuning key 8: column splits of a tile in the expand
     const int32_t nblk = (AP.tv.d_out + 63) / 64;
@@ -778,19 +801,14 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
     P.moff_perm = (int32_t)L.perm;
     P.moff_desc = (int32_t)L.tile_desc;
     P.target_rows = pool->r_max;
-    P.list = reinterpret_cast<int32_t *>((char *)workspace + ws_partials);
-    P.list_cap = max_long;
+    P.list = const_cast<int32_t *>(AP.meta) + L.long_list;
+    P.list_cap = L.cap_tile;
     P.shrink_grid = 2 * pool->sm_count;   // two blocks fit on an SM: the grid fills the GPU exactly once
     if (check_only) {   // nothing has been launched: the caller only asks whether the path applies
         *handled = true;
         return LORA_OK;
     }
-    const int32_t units = max_long;   // block columns: one per work-list entry, the unused ones leave at once
-    tc_worklist_kernel<<<1, 256, 0, stream>>>(P);
-    {
-        lora_status_t sl = count_launch();
-        if (sl != LORA_OK) return sl;
-    }
+    const int32_t units = max_long;   // block columns of the expand: one per list entry, the unused ones leave at once
 
     P.y = AP.y;
     P.ldy = AP.ldy;

@@ -73,7 +73,7 @@ enum { H_T = 0, H_NACTIVE = 1, H_NINVALID = 2, H_NSEG = 3, H_NTILE = 4, H_TILE_M
 struct MetaLayout {
     int32_t cap_seg, cap_tile;
     int64_t perm, seg_slot, seg_start, seg_rank, seg_flags, tile_seg, tile_row0, tile_rows,
-        tile_flags, tile_desc, unit_desc, unit_perm, words;
+        tile_flags, tile_desc, unit_desc, unit_perm, long_list, words;
     int32_t cap_unit;
 };
 
@@ -100,6 +100,10 @@ __host__ __device__ inline MetaLayout meta_layout(int32_t T, int32_t num_slots, 
     L.cap_unit = L.cap_tile * ((tile_m + 15) / 16);
     L.unit_desc = o;  o += 4 * (int64_t)L.cap_unit;
     L.unit_perm = o;  o += 16 * (int64_t)L.cap_unit;
+    // Tiles for the tensor-core kernels of lora_sgmv_apply (runs of consecutive tokens), in tile
+    // order: [0] = their number, then their tile numbers.  Written after the build when the batch
+    // qualifies for those kernels, else left alone.
+    L.long_list = o;  o += ((int64_t)L.cap_tile + 1 + 3) & ~(int64_t)3;
     L.words = o;
     return L;
 }
@@ -163,16 +167,22 @@ struct lora_pool {
         const void *ptr;
         int32_t T, tile_m, long_min;
         bool fresh;   // built, and no apply has been queued behind the build yet
+        bool has_list;   // the list of long tiles was written behind the build
     };
     std::vector<MetaRecord> metas;
-    void remember_meta(const void *ptr, int32_t T, int32_t tile_m, int32_t long_min) {
+    void remember_meta(const void *ptr, int32_t T, int32_t tile_m, int32_t long_min, bool has_list) {
         for (MetaRecord &m : metas)
             if (m.ptr == ptr) {
-                m.T = T; m.tile_m = tile_m; m.long_min = long_min; m.fresh = true;
+                m.T = T; m.tile_m = tile_m; m.long_min = long_min; m.fresh = true; m.has_list = has_list;
                 return;
             }
         if (metas.size() >= 256) metas.erase(metas.begin());
-        metas.push_back({ptr, T, tile_m, long_min, true});
+        metas.push_back({ptr, T, tile_m, long_min, true, has_list});
+    }
+    bool meta_has_list(const void *ptr) const {
+        for (const MetaRecord &m : metas)
+            if (m.ptr == ptr) return m.has_list;
+        return false;
     }
     bool find_meta(const void *ptr, int32_t T, int32_t *tile_m) const {
         for (const MetaRecord &m : metas)

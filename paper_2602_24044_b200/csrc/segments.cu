@@ -6,7 +6,7 @@
 // its prefix sums (O(T + N) integer work from L2), then each warp owns whole slots and writes
 // that slot's run of `perm` by scanning the token list in order with warp ballots, which makes
 // the order inside a run ascending by construction.
-#include "common.cuh"
+#include "apply_common.cuh"
 
 namespace lora {
 
@@ -537,7 +537,11 @@ lora_status_t lora_build_segments(lora_pool_t *pool, const int32_t *slot_idx_dev
     if (!guard.ok) return cuda_fail(cudaErrorInvalidDevice);
     lora_status_t s = launch_build_segments(pool, slot_idx_dev, T, tile_m, long_min, meta_dev,
                                             (cudaStream_t)stream);
-    if (s == LORA_OK) pool->remember_meta(meta_dev, T, tile_m, long_min);
+    // batches that lora_sgmv_apply gives to its tensor-core kernels: the list of their tiles, once
+    // per build (tuning key 4 is read here)
+    const bool with_list = s == LORA_OK && tc_path_wanted(pool, T, tile_m);
+    if (with_list) s = launch_tc_worklist(pool, T, tile_m, meta_dev, (cudaStream_t)stream);
+    if (s == LORA_OK) pool->remember_meta(meta_dev, T, tile_m, long_min, with_list);
     return s;
 }
 
