@@ -85,6 +85,7 @@ def test_segments_bytes_matches_documented_layout():
     desc_end = words
     cap_unit = cap_tile * ((tile_m + 15) // 16)          # 16-row pieces of all tiles
     words += 4 * cap_unit + 16 * cap_unit                # library-private unit records and row ids
+    words += (cap_tile + 1 + 3) // 4 * 4                 # library-private list of long tiles
     assert lb.segments_bytes(T, N, tile_m) == 4 * words
     assert lb.segments_bytes(0, N, tile_m) == 4 * 20
     with pytest.raises(lb.LoraError):
