@@ -87,7 +87,7 @@ def test_segments_bytes_matches_documented_layout():
     words += 4 * cap_unit + 16 * cap_unit                # library-private unit records and row ids
     words += (cap_tile + 1 + 3) // 4 * 4                 # library-private list of long tiles
     assert lb.segments_bytes(T, N, tile_m) == 4 * words
-    assert lb.segments_bytes(0, N, tile_m) == 4 * 20
+    assert lb.segments_bytes(0, N, tile_m) == 4 * 24      # header, seg_start[1], padding, list count
     with pytest.raises(lb.LoraError):
         lb.segments_bytes(-1, N, tile_m)
     meta = np.arange(words, dtype=np.int32)
