@@ -152,7 +152,8 @@ static lora_status_t launch_h(lora_pool_t *pool, FusedParams &P, int32_t C, cons
     int32_t S = pool->tuning[5];
     if (S < 2 || S > MAX_STAGES) S = 2;   // two stages and more resident blocks beat deeper rings
     int32_t o = SM_HEADER;
-    P.off_part = o;   o += mrows * 64 * 4;
+    const int32_t nwc = H == 2 ? 8 : 4;   // consumer warps of the kernel
+    P.off_part = o;   o += mrows * 16 * nwc * 4;
     // general kernel: a block's partial stays in its own shared memory, two sets (the decode kernel
     // pushes partials into every block; its carve-up is fixed)
     P.push = 0;
@@ -181,7 +182,7 @@ static lora_status_t launch_h(lora_pool_t *pool, FusedParams &P, int32_t C, cons
         lc.attr_smem = smem;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.blockDim = dim3(FT_ALL, 1, 1);
+    cfg.blockDim = dim3((unsigned)(32 * (nwc + 1)), 1, 1);
     cfg.dynamicSmemBytes = (size_t)smem;
     cfg.stream = stream;
     cudaLaunchAttribute at[2];

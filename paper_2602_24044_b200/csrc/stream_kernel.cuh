@@ -33,7 +33,7 @@ constexpr int SM_XB = 64;        // two mbarriers: every block has published its
 constexpr int SM_YB = 80;        // two mbarriers: every block has read the partials
 constexpr int SM_FLAG = 96;      // int32: a bounded wait of this block has expired
 constexpr int SM_COUNT = 100;    // int32: jobs requested so far
-constexpr int SM_CBAR = 104;     // mbarrier: the 128 consumer threads meet (bounded, unlike bar.sync)
+constexpr int SM_CBAR = 104;     // mbarrier: the consumer threads meet (bounded, unlike bar.sync)
 constexpr int SM_JOB = 128;      // job headers, 16 bytes per stage
 constexpr int SM_UNIT = 192;     // unit entries, ring of eight
 constexpr int UNIT_ENTRIES = 8;
@@ -295,7 +295,7 @@ struct CLane {
 };
 
 // One shrink chunk: acc += x[rows, chunk] . A_i[chunk, 16 ranks of this warp].  RP: rank bucket; H: 1
-// when a unit holds at most 8 rows, 2 when rows 8..15 can be occupied.  The four warps split the
+// when a unit holds at most 8 rows, 2 when rows 8..15 can be occupied.  The NWC consumer warps split the
 // rank tiles WN ways and the chunk's 64-column blocks WK ways: every warp owns two rank tiles of 8
 // and every WK-th column block.  Operand fragments come by ldmatrix; lane l names row (l & 7) of 8x8 matrix
 // (l >> 3):
@@ -303,10 +303,10 @@ struct CLane {
 //            n sits at n * 128 bytes of the column block, its 16-byte chunk c at ((c ^ (n & 7)) << 4);
 //            the even part of c is folded in per step with one XOR
 //   tokens:  (rows 0-7, k 0-7) (rows 8-15, k 0-7) (rows 0-7, k 8-15) (rows 8-15, k 8-15)
-template <int RP, int H>
+template <int RP, int H, int NWC>
 __device__ __forceinline__ void shrink_job(const CLane &L, uint32_t w_stage, uint32_t t_stage, int32_t ncols,
                                            uint32_t blk_bytes, float (&acc)[2][4]) {
-    constexpr int WN = RP / 16, WK = 4 / WN;
+    constexpr int WN = RP / 16, WK = NWC / WN;   // a warp whose column block the job does not have stays idle
     constexpr int NB = chunk_cols(RP == 16 ? 0 : RP == 32 ? 1 : 2) / 64;   // column blocks of a job
     constexpr bool hi_rows = H == 2;
     const int wk = L.warp % WK, wn = L.warp / WK;
@@ -351,10 +351,10 @@ struct XUnit {
 // One expand chunk: y[rows, chunk] = y_base + s * v . B_i[ranks, chunk] for this warp's columns.
 // B_i fragments by ldmatrix (transposing): lane l names rank row ks + 8 (mi & 1) + r of column tile
 // 2 np + (mi >> 1); v fragments (high and low bf16 parts) by ldmatrix from the block's copies.
-template <int RP, int H>
+template <int RP, int H, int NWC>
 __device__ __forceinline__ void expand_job(const CLane &L, uint32_t w_stage, uint32_t t_stage, uint32_t vh,
                                            uint32_t vl, int32_t ncols, int32_t c, const XUnit &xu) {
-    constexpr int CW = chunk_cols(RP == 16 ? 0 : RP == 32 ? 1 : 2), NW = CW / 4, NP = NW / 16, KT = RP / 16;
+    constexpr int CW = chunk_cols(RP == 16 ? 0 : RP == 32 ? 1 : 2), NW = CW / NWC, NP = NW / 16, KT = RP / 16;
     constexpr bool hi_rows = H == 2;
     const int32_t nc = ncols - L.warp * NW;   // columns of this warp's share
     if (nc <= 0) return;
@@ -427,6 +427,7 @@ template <int H>
 __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *smem, int32_t cid, int32_t G,
                                           uint32_t crank, uint32_t csize) {
     constexpr int mrows = 8 * H;
+    constexpr int NWC = 4 * H, CT = 32 * NWC, LOG_NWC = H == 2 ? 3 : 2;   // consumer warps, threads
     CLane L;
     L.tid = threadIdx.x; L.lane = L.tid & 31; L.warp = L.tid >> 5; L.g = L.lane >> 2; L.t = L.lane & 3;
     L.mi = L.lane >> 3; L.r = L.lane & 7;
@@ -434,7 +435,7 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + SM_FULL);
     uint64_t *empty = reinterpret_cast<uint64_t *>(smem + SM_EMPTY);
     volatile int32_t *dead = reinterpret_cast<volatile int32_t *>(smem + SM_FLAG);
-    float *part = reinterpret_cast<float *>(smem + P.off_part);     // [WK][mrows][RP] = mrows x 64 floats
+    float *part = reinterpret_cast<float *>(smem + P.off_part);     // [WK][mrows][RP] = mrows x 16 NWC floats
     __nv_bfloat16 *Vh = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_vh);   // [mrows][PV]
     __nv_bfloat16 *Vl = reinterpret_cast<__nv_bfloat16 *>(smem + P.off_vl);
     const uint32_t w_base = smem_u32(smem + P.off_w), t_base = smem_u32(smem + P.off_tok);
@@ -476,7 +477,7 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
             const FusedItem &it = P.item[job.y];
             const __nv_bfloat16 *src = it.yb + (int64_t)job.z * it.ldyb;
             __nv_bfloat16 *dst = it.y + (int64_t)job.z * it.ldy;
-            for (int32_t v = (int32_t)crank * FT + tid; v < it.d_out / 8; v += (int32_t)csize * FT)
+            for (int32_t v = (int32_t)crank * CT + tid; v < it.d_out / 8; v += (int32_t)csize * CT)
                 reinterpret_cast<uint4 *>(dst)[v] = ldg16(src + (int64_t)v * 8);
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[st]);
@@ -488,15 +489,15 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
 #pragma unroll
                 for (int i = 0; i < 2; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.0f;
             }
-            if (sh == 0) shrink_job<16, H>(L, w_stage, t_stage, job.w, blk_bytes, acc);
-            else if (sh == 1) shrink_job<32, H>(L, w_stage, t_stage, job.w, blk_bytes, acc);
-            else shrink_job<64, H>(L, w_stage, t_stage, job.w, blk_bytes, acc);
+            if (sh == 0) shrink_job<16, H, NWC>(L, w_stage, t_stage, job.w, blk_bytes, acc);
+            else if (sh == 1) shrink_job<32, H, NWC>(L, w_stage, t_stage, job.w, blk_bytes, acc);
+            else shrink_job<64, H, NWC>(L, w_stage, t_stage, job.w, blk_bytes, acc);
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[st]);
             if (job.x & J_LAST) {
                 // ---- the block's partial is made available to the cluster (buffer set kp & 1) ----
                 const int b = kp & 1;
-                const int RP = 16 << sh, WK = 4 >> sh;
+                const int RP = 16 << sh, WK = NWC >> sh;
                 if (kp >= 2) {   // the peers have read what this set held two units ago
                     ok = __all_sync(0xffffffffu, mbar_wait_cluster(reinterpret_cast<uint64_t *>(smem + SM_YB) + b,
                                                                    (uint32_t)((kp - 2) >> 1) & 1u));
@@ -505,7 +506,7 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
                         break;
                     }
                 }
-                const int wk = L.warp & (WK - 1), wn = L.warp >> (2 - sh);
+                const int wk = L.warp & (WK - 1), wn = L.warp >> (LOG_NWC - sh);
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
                     float *p0 = part + (wk * mrows + L.g) * RP + (wn * 2 + i) * 8 + 2 * L.t;
@@ -515,7 +516,7 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
                 if (!meet()) { ok = false; break; }
                 // block partial: the column blocks' sums in order
                 float *vbuf = reinterpret_cast<float *>(smem + P.off_vpart + b * P.vbuf_bytes);
-                for (int i = tid; i < mrows * RP; i += FT) {
+                for (int i = tid; i < mrows * RP; i += CT) {
                     if ((i >> (4 + sh)) < rows) {
                         float v = part[i];
                         for (int w = 1; w < WK; ++w) v += part[w * mrows * RP + i];
@@ -550,7 +551,7 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
                 // the previous unit's expand chunks have read their last fragment of v
                 if (!meet()) { ok = false; break; }
                 const uint32_t vp_addr = smem_u32(smem + P.off_vpart + b * P.vbuf_bytes);
-                for (int i = tid; i < rows * rank16; i += FT) {
+                for (int i = tid; i < rows * rank16; i += CT) {
                     const int m = i / rank16, k = i - m * rank16;
                     float v = 0.0f;
                     if (k < rank) {
@@ -571,7 +572,7 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
                 if (tid < (int)csize) mbar_arrive_peer(reinterpret_cast<uint64_t *>(smem + SM_YB) + b, (uint32_t)tid);
                 ++kr;
                 const FusedItem &it = P.item[ue->item];
-                const int NW = chunk_cols(sh) / 4;
+                const int NW = chunk_cols(sh) / NWC;
                 xu.row0 = L.g < rows;
                 xu.row1 = H == 2 && L.g + 8 < rows;
                 xu.y0 = it.y + (int64_t)(xu.row0 ? ue->rowid[L.g] : 0) * it.ldy + ue->b_lo + L.warp * NW + 2 * L.t;
@@ -581,9 +582,9 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
                 xu.blk_bytes = (uint32_t)ue->rb * 128u;
                 xu.rank16 = rank16;
             }
-            if (sh == 0) expand_job<16, H>(L, w_stage, t_stage, vh_addr, vl_addr, job.w, job.z, xu);
-            else if (sh == 1) expand_job<32, H>(L, w_stage, t_stage, vh_addr, vl_addr, job.w, job.z, xu);
-            else expand_job<64, H>(L, w_stage, t_stage, vh_addr, vl_addr, job.w, job.z, xu);
+            if (sh == 0) expand_job<16, H, NWC>(L, w_stage, t_stage, vh_addr, vl_addr, job.w, job.z, xu);
+            else if (sh == 1) expand_job<32, H, NWC>(L, w_stage, t_stage, vh_addr, vl_addr, job.w, job.z, xu);
+            else expand_job<64, H, NWC>(L, w_stage, t_stage, vh_addr, vl_addr, job.w, job.z, xu);
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[st]);
             if (job.x & J_FINAL) break;
@@ -618,12 +619,12 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
             const int32_t per_blk = (vecs + (int32_t)csize - 1) / (int32_t)csize;
             const int32_t v_lo = (int32_t)crank * per_blk, v_n = max(0, min(per_blk, vecs - v_lo));
             const int32_t total = rows * v_n;
-            for (int32_t i0 = tid; i0 < total; i0 += 4 * FT) {
+            for (int32_t i0 = tid; i0 < total; i0 += 4 * CT) {
                 uint4 val[4];
                 int64_t off[4];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    const int32_t i = i0 + q * FT;
+                    const int32_t i = i0 + q * CT;
                     const int32_t m = i < total ? i / v_n : 0, v = i < total ? v_lo + i - m * v_n : 0;
                     off[q] = (int64_t)rowidx[m];
                     val[q] = make_uint4(0, 0, 0, 0);
@@ -632,7 +633,7 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
                 }
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
-                    if (i0 + q * FT < total) *reinterpret_cast<uint4 *>(it.y + off[q]) = val[q];
+                    if (i0 + q * CT < total) *reinterpret_cast<uint4 *>(it.y + off[q]) = val[q];
             }
         }
     }
@@ -641,8 +642,11 @@ __device__ __forceinline__ void consumers(const FusedParams &P, unsigned char *s
 }  // namespace gen
 
 // H: 1 when a unit holds at most 8 rows (decode tiles, single tokens), 2 otherwise.
+// Four consumer warps at H = 1, eight at H = 2 (a 16-row job is twice the work, and the batches that
+// come here keep few blocks per SM: the launch is bound by the consumer warps' own chains), plus
+// the requesting warp.
 template <int H>
-__global__ void __launch_bounds__(FT_ALL, LORA_FUSED_MIN_BLOCKS)
+__global__ void __launch_bounds__(32 * (4 * H + 1), H == 2 ? 3 : LORA_FUSED_MIN_BLOCKS)
 stream_kernel(const __grid_constant__ FusedParams P) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t csize = cluster_nctarank(), crank = cluster_ctarank();
@@ -659,19 +663,20 @@ stream_kernel(const __grid_constant__ FusedParams P) {
         griddep_wait();
         return;
     }
-    if (warp == 4 && lane < MAPS_PER_TARGET) prefetch_tensormap(P.maps + P.item[0].map_base + lane);
+    constexpr int NWC = 4 * H;   // consumer warps; warp NWC requests the jobs
+    if (warp == NWC && lane < MAPS_PER_TARGET) prefetch_tensormap(P.maps + P.item[0].map_base + lane);
     if (tid == 0) {
         uint64_t *full = reinterpret_cast<uint64_t *>(smem + gen::SM_FULL);
         uint64_t *empty = reinterpret_cast<uint64_t *>(smem + gen::SM_EMPTY);
         for (int s = 0; s < P.n_stages; ++s) {
             mbar_init(&full[s], 1);
-            mbar_init(&empty[s], 4);
+            mbar_init(&empty[s], NWC);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(reinterpret_cast<uint64_t *>(smem + gen::SM_XB) + b, csize);
             mbar_init(reinterpret_cast<uint64_t *>(smem + gen::SM_YB) + b, csize);
         }
-        mbar_init(reinterpret_cast<uint64_t *>(smem + gen::SM_CBAR), FT);
+        mbar_init(reinterpret_cast<uint64_t *>(smem + gen::SM_CBAR), 32 * NWC);
         *reinterpret_cast<int32_t *>(smem + gen::SM_FLAG) = 0;
         *reinterpret_cast<int32_t *>(smem + gen::SM_COUNT) = 0;
         fence_mbar_init();
@@ -685,7 +690,7 @@ stream_kernel(const __grid_constant__ FusedParams P) {
     // complete before the preceding kernel started when P.early is set (the host sets it only
     // then), so they are read, and the first weight tiles requested, ahead of the wait.
     if (!P.early) griddep_wait();
-    if (warp == 4) {
+    if (warp == NWC) {
         gen::producer(P, smem, cid, G, crank, lane);
         cluster_wait();     // the opening barrier (this warp touches no peer)
         cluster_arrive();   // the closing one
