@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None: no capture of the current kernel on that workload)
-NCU_TRAFFIC = {1: 22.9e6, (4, "layer"): 269.7e6, 3: 172.0e6}
+NCU_TRAFFIC = {1: 22.9e6, (4, "layer"): 269.7e6, 3: 171.1e6}
 
 PAPER_CONTEXT = {
     "note": "system-level results of the paper, other hardware, context only",
