@@ -52,6 +52,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=160)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=200)
+    ap.add_argument("--e2e-lanes", type=int, default=3, help="streams (with their staging buffers) the end-to-end steps rotate over")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--algo", type=int, default=None,
                     help="apply path: 0 fused cluster kernel (default), 1 two-phase kernels")
@@ -644,15 +645,16 @@ def main():
     d_in0, d_out0 = wl.targets[wl.calls[0]]
     Ke = args.e2e_steps if cfg in (0, 1) else max(3, min(args.e2e_steps, 10))
     x_h, yb_h = wl.activations(0)
-    xh = [bf16_tensor(x_h, pin=True) for _ in range(2)]
-    ybh = [bf16_tensor(yb_h, pin=True) for _ in range(2)]
-    yh = [torch.empty((T, d_out0), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+    NL = args.e2e_lanes
+    xh = [bf16_tensor(x_h, pin=True) for _ in range(NL)]
+    ybh = [bf16_tensor(yb_h, pin=True) for _ in range(NL)]
+    yh = [torch.empty((T, d_out0), dtype=torch.bfloat16).pin_memory() for _ in range(NL)]
     sh = torch.from_numpy(wl.slot_idx.copy()).pin_memory()
     tp0, xd0, ybd0, yd0 = sets[0][0]
-    # two lanes (stream + device staging buffers each), used alternately: the host-to-device copy of
-    # one step overlaps the device-to-host copy of the step before it
+    # lanes (stream + device staging buffers each), used in turn: the host-to-device copy of one
+    # step overlaps the compute and the device-to-host copy of the steps before it
     lanes = []
-    for lane in range(2):
+    for lane in range(NL):
         lanes.append({
             "stream": s.compute if lane == 0 else torch.cuda.Stream(dev),
             "x": xd0 if lane == 0 else torch.empty_like(xd0),
@@ -664,7 +666,7 @@ def main():
         })
 
     def e2e_step(i):
-        c = i % 2
+        c = i % NL
         L = lanes[c]
         lb.apply_host(s.pool, tp0, 1 if sgmv else 0, xh[c], ybh[c], yh[c], sh, T, wl.tile_m, wl.long_min,
                       L["x"], L["yb"], L["y"], L["sidx"], L["meta"], L["ws"], L["stream"])
@@ -738,7 +740,7 @@ def main():
         },
         "step_GBps": alg / (ms / K * 1e-3) / 1e9,
         "e2e": {"value": whole_job_value(world, T, Ke, e2e_s * 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "api": "lora_apply_host (first projection of the step), two streams used alternately",
+                "d2h_bytes_per_step": d2h, "api": "lora_apply_host (first projection of the step), %d streams used in turn" % NL,
                 "steps": Ke},
         "gpu_launches": int(launches),
         "device_status_words": status_words,
