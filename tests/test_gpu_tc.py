@@ -123,3 +123,19 @@ def test_prefill_apply_in_a_cuda_graph():
                 g.replay()
             assert np.array_equal(bf16_bits(y), eager)
         assert s.status()[1] == 0
+
+
+def test_leftover_tiles_beside_or_after_the_tensor_core_kernels_give_the_same_bits():
+    """The tiles the tensor-core kernels leave over run on the pool's own stream beside them
+    (default) or after them on the caller's stream (tuning key 6 = 1): disjoint rows, same result."""
+    rng = np.random.default_rng(58)
+    dec = rng.integers(0, 10, 120)
+    slot_idx = np.concatenate([np.repeat([1, 4], 260), dec, np.repeat([4], 70), np.repeat([8], 150)]).astype(np.int32)
+    wl = W.make_custom(0, 1536, 1024, 10, [8, 16, 32], kind="sgmv", tile_m=128, scale=1.2,
+                       weight_mode="unitB", slot_idx=slot_idx, frac_none=0.03, seed=58)
+    y_ref, _ = oracle_full(wl)
+    y_beside, n_beside = _run(wl)
+    y_after, n_after = _run(wl, tuning={4: 2, 6: 1})
+    check_tolerance(y_beside, y_ref, what="beside")
+    assert np.array_equal(y_beside, y_after)
+    assert n_beside == n_after
