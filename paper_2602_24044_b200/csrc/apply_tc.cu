@@ -160,7 +160,8 @@ __host__ __device__ constexpr uint32_t instr_desc(uint32_t M, uint32_t N, uint32
 }
 }  // namespace tc
 
-constexpr int TCX_THREADS = 192;   // expand: four epilogue warps, one warp that issues MMAs, one that issues copies
+constexpr int XQ = 2;               // expand: epilogue warps per quarter of the rows (each takes 64 / XQ columns; 1: 561, 2: 553, 4: 557 us per prefill step)
+constexpr int TCX_THREADS = 32 * (4 * XQ + 2);   // plus one warp that issues MMAs and one that issues copies
 constexpr int TC_ROWS = 128;       // rows of a long tile
 constexpr int SH_STAGES = 3;       // shrink: ring of (x tile, A tile) stages
 constexpr int XT_BYTES = TC_ROWS * 128;   // 128 rows x 64 bf16
@@ -487,12 +488,12 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
         for (int s = 0; s < S; ++s) {
             tc::mbar_init(&full[s], 1);
             tc::mbar_init(&mma_done[s], 1);
-            tc::mbar_init(&epi_done[s], TC_ROWS);
+            tc::mbar_init(&epi_done[s], XQ * TC_ROWS);
         }
         *failed = 0;
         tc::fence_mbar_init();
     }
-    if (warp == 4) {
+    if (warp == 4 * XQ) {
         tc::tmem_alloc(tmem_slot, C::TMEM_COLS);
         tc::tmem_relinquish();
     }
@@ -563,7 +564,7 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
         return true;
     };
 
-    if (warp == 4) {
+    if (warp == 4 * XQ) {
         // ---- one thread issues each block's MMAs as soon as its tiles have landed; it only ever
         // waits for data --------------------------------------------------------------------------
         if (lane == 0) {
@@ -572,7 +573,7 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
             }
         }
         __syncwarp();
-    } else if (warp == 5) {
+    } else if (warp == 4 * XQ + 1) {
         // ---- one thread owns the stages' life cycle: it requests the first S blocks, and whenever
         // the epilogue has finished a block it sends the tile out (TMA store), waits until the
         // store has read the stage and requests the block that reuses it.  Every stage that is not
@@ -604,29 +605,33 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
         }
         __syncwarp();
     } else {
-        // ---- epilogue warps: thread = row; the y_base tile (128-byte swizzle) is updated in place
-        const int m = warp * 32 + lane;
+        // ---- epilogue warps: XQ per quarter of the rows (a warp reads the tensor-memory lanes of
+        // its number modulo four), each taking 64 / XQ of the block's columns; the y_base tile
+        // (128-byte swizzle) is updated in place
+        const int quarter = warp & 3, part = warp >> 2;
+        const int m = quarter * 32 + lane;
         for (int32_t j = 0; j < nblk; ++j) {
             const int s = j % S;
-            // all four warps take the same decision (a thread that left alone would strand the
+            // all eight warps take the same decision (a thread that left alone would strand the
             // others at the named barrier below)
             const uint32_t bad = (*failed != 0 || !tc::mbar_wait(&mma_done[s], (uint32_t)(j / S) & 1u)) ? 1u : 0u;
             uint32_t any_bad;
             asm volatile(
                 "{\n\t.reg .pred p, q;\n\t"
                 "setp.ne.u32 p, %1, 0;\n\t"
-                "bar.red.or.pred q, 1, 128, p;\n\t"
+                "bar.red.or.pred q, 1, %2, p;\n\t"
                 "selp.u32 %0, 1, 0, q;\n\t}"
                 : "=r"(any_bad)
-                : "r"(bad)
+                : "r"(bad), "n"(XQ * TC_ROWS)
                 : "memory");
             if (any_bad) { ok = false; *failed = 1; break; }
             tc::tc_fence_after();
             unsigned char *tile = stages + s * C::STAGE;
 #pragma unroll
-            for (int c = 0; c < 64; c += 16) {
+            for (int cc = 0; cc < 64 / XQ; cc += 16) {
+                const int c = part * (64 / XQ) + cc;
                 uint32_t r[16];
-                tc::tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + s * 64 + c, r);
+                tc::tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + s * 64 + c, r);
                 tc::tmem_ld_wait();
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
@@ -645,7 +650,7 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
                 if (m < lt.rows) {
                     __nv_bfloat16 *yrow = P.y + (int64_t)(lt.t0 + m) * P.ldy + colb;
 #pragma unroll
-                    for (int chunk = 0; chunk < 8; ++chunk)
+                    for (int chunk = part * (8 / XQ); chunk < (part + 1) * (8 / XQ); ++chunk)
                         if (colb + chunk * 8 < P.tv.d_out)
                             *reinterpret_cast<uint4 *>(yrow + chunk * 8) =
                                 *reinterpret_cast<const uint4 *>(tile + m * 128 + ((chunk ^ (m & 7)) << 4));
@@ -653,13 +658,13 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
             } else {
                 tc::fence_proxy_async();    // the tile is read by the TMA store
             }
-            tc::mbar_arrive(&epi_done[s]);  // 128 arrivals: every row of the stage is finished
+            tc::mbar_arrive(&epi_done[s]);  // every epilogue thread: all rows and columns of the stage are finished
         }
     }
     if (tid == 0 && *failed) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
     tc::tc_fence_before();
     __syncthreads();
-    if (warp == 4) tc::tmem_dealloc(tmem, C::TMEM_COLS);
+    if (warp == 4 * XQ) tc::tmem_dealloc(tmem, C::TMEM_COLS);
 }
 
 // ---------------------------------------------------------------------------------------------
