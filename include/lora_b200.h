@@ -179,7 +179,7 @@ lora_status_t lora_pool_selftest_wait_expiry(lora_pool_t *pool, int32_t polls, i
  *   key 6  lora_sgmv_apply: 1 = the tiles the tensor-core kernels leave over run after them on the
  *          caller's stream, not beside them on the pool's own stream
  *   key 7  segment builder: 1 = one warp per slot also for long batches
- *   key 8  tensor-core expand of lora_sgmv_apply: blocks a tile's columns are split over (0 = automatic)
+ *   key 8  tensor-core expand of lora_sgmv_apply: blocks per SM in its grid (0 = the default, 8)
  *   key 9  fused kernel: share (1 .. 99 %) of the resident clusters one launch may take
  *   key 10 1 = decode batches take the general fused kernel, not the decode kernel
  *   key 11 when a fused kernel lets its successor on the stream become resident: 1 = only at its

@@ -171,7 +171,8 @@ struct TcParams {
     TargetView tv;
     const int32_t *meta;
     float *ws;              // [KS][T][RS] fp32 partial v: one slab per piece of a tile
-    int32_t T, RS, KS, NS;  // KS: slabs the workspace holds
+    int32_t T, RS, KS;      // KS: slabs the workspace holds
+    int32_t expand_grid;    // blocks of the expand launch
     int32_t shrink_grid;    // blocks of the shrink launch (fixes how the walk is cut into pieces)
     int32_t moff_perm, moff_desc;
     int32_t target_rows;    // r_max: rows of a slot's matrices
@@ -455,6 +456,9 @@ struct ExpandCfg {
     static constexpr uint32_t TMEM_COLS = STAGES <= 2 ? 128 : STAGES <= 4 ? 256 : 512;  // ring of 64-column accumulators
 };
 
+// The expand walks the (long tile, 64-column block of d_out) pairs in tile order, cut into equal
+// spans like the shrink's walk, one span per block; the grid is several waves of blocks.  A block
+// whose span crosses into the next tile builds that tile's v when it gets there.
 template <int RP>
 __global__ void __launch_bounds__(TCX_THREADS)
 tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
@@ -471,18 +475,20 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
     uint64_t *full = reinterpret_cast<uint64_t *>(Vl + C::V_BYTES);
     uint64_t *mma_done = full + S;
     uint64_t *epi_done = mma_done + S;  // every epilogue thread has finished its row of the stage
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(epi_done + S);
+    uint64_t *v_ready = epi_done + S;   // the tile's v (both bf16 parts) is in shared memory
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(v_ready + 1);
     volatile int32_t *failed = reinterpret_cast<volatile int32_t *>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const LongTile lt = long_tile(P, blockIdx.x);
-    if (!lt.ok) return;
-    // 64-column blocks of d_out owned by this block
-    const int32_t nblk_all = (P.tv.d_out + 63) / 64;
-    const int32_t per = (nblk_all + P.NS - 1) / P.NS;
-    const int32_t b0 = min((int32_t)blockIdx.y * per, nblk_all), b1 = min(b0 + per, nblk_all);
-    const int32_t nblk = b1 - b0;
-    if (nblk <= 0) return;
+    const int32_t n_long = P.list[0];
+    if (n_long <= 0) return;
+    const int32_t nblk = (P.tv.d_out + 63) / 64;            // column blocks of one tile
+    const int64_t total = (int64_t)n_long * nblk;
+    // at least 16 column blocks per block: every span starts by building its tile's v
+    const int64_t span = max((total + gridDim.x - 1) / gridDim.x, (int64_t)16);
+    const int64_t g0 = (int64_t)blockIdx.x * span, g1 = min(g0 + span, total);
+    if (g0 >= g1) return;
+    const ShrinkSplit sp = shrink_split(n_long, P.tv.d_in, P.KS, P.shrink_grid);
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
@@ -490,6 +496,7 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
             tc::mbar_init(&mma_done[s], 1);
             tc::mbar_init(&epi_done[s], XQ * TC_ROWS);
         }
+        tc::mbar_init(v_ready, XQ * TC_ROWS);
         *failed = 0;
         tc::fence_mbar_init();
     }
@@ -497,80 +504,45 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
         tc::tmem_alloc(tmem_slot, C::TMEM_COLS);
         tc::tmem_relinquish();
     }
-    // v = sum of the tile's pieces (in order); thread = row.  Stored as bf16 high and low parts
-    // in the no-swizzle K-major layout: 8 x 8 core matrices of 128 bytes, the core matrix of row
-    // group mg and rank group kg at (kg * 16 + mg) * 128 bytes.
-    const ShrinkSplit sp = shrink_split(P.list[0], P.tv.d_in, P.KS, P.shrink_grid);
-    const int32_t n_pieces = last_block_of(sp, (int32_t)blockIdx.x) - first_block_of(sp, (int32_t)blockIdx.x) + 1;
-    if (tid < TC_ROWS) {
-        const int32_t m = tid;
-        const float *src = P.ws + ((int64_t)lt.row0 + m) * P.RS;
-        const int64_t ks_stride = (int64_t)P.T * P.RS;
-#pragma unroll
-        for (int kg = 0; kg < RP / 8; ++kg) {
-            float v[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) v[e] = 0.0f;
-            for (int32_t q = 0; q < n_pieces && m < lt.rows; ++q) {   // rows past a short tile's end stay zero
-                const float4 a = *reinterpret_cast<const float4 *>(src + q * ks_stride + kg * 8);
-                const float4 b = *reinterpret_cast<const float4 *>(src + q * ks_stride + kg * 8 + 4);
-                v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
-                v[4] += b.x; v[5] += b.y; v[6] += b.z; v[7] += b.w;
-            }
-            uint32_t hi[4], lo[4];
-#pragma unroll
-            for (int e = 0; e < 8; e += 2) {
-                const float v0 = kg * 8 + e < lt.rank ? v[e] : 0.0f;
-                const float v1 = kg * 8 + e + 1 < lt.rank ? v[e + 1] : 0.0f;
-                const __nv_bfloat16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
-                hi[e / 2] = pack2(__bfloat162float(h0), __bfloat162float(h1));
-                lo[e / 2] = pack2(v0 - __bfloat162float(h0), v1 - __bfloat162float(h1));
-            }
-            const int off = (kg * 16 + (m >> 3)) * 128 + (m & 7) * 16;
-            *reinterpret_cast<uint4 *>(Vh + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-            *reinterpret_cast<uint4 *>(Vl + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-        }
-    }
-    tc::fence_proxy_async();     // v was written with ordinary stores and is read by the MMA unit
     tc::tc_fence_before();
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    bool ok = true;
 
     constexpr uint32_t IDESC = tc::instr_desc(128, 64, 0, 1);   // A = v (K-major), B = B_i tile (N-major)
-    auto issue_load = [&](int32_t j) {
-        const int s = j % S;
-        unsigned char *st = stages + s * C::STAGE;
-        tc::mbar_expect_tx(&full[s], XT_BYTES + C::BT_BYTES);
-        tc::tma_load_2d(st, &map_yb, (b0 + j) * 64, lt.t0, &full[s]);
-        tc::tma_load_3d(st + XT_BYTES, &map_b, (b0 + j) * 64, 0, lt.slot, &full[s]);
-    };
-    auto issue_mma = [&](int32_t j) -> bool {
-        const int s = j % S;
-        if (!tc::mbar_wait(&full[s], (uint32_t)(j / S) & 1u)) return false;
-        tc::tc_fence_after();
-        const uint32_t ba = tc::smem_u32(stages + s * C::STAGE + XT_BYTES);
-        const uint32_t vh = tc::smem_u32(Vh), vl = tc::smem_u32(Vl);
-        const int32_t ksteps = (lt.rank + 15) >> 4;
-        for (int32_t k = 0; k < ksteps; ++k) {
-            // v: two rank groups per step, 2048 bytes apart; B tile: 16 rank rows = 2048 bytes per step
-            const uint64_t bd = tc::smem_desc(ba + k * 2048, 16, 1024, tc::LAYOUT_SW128);
-            tc::umma(tmem + s * 64, tc::smem_desc(vh + k * 4096, 2048, 128, tc::LAYOUT_NONE), bd, IDESC,
-                     k > 0 ? 1u : 0u);
-            tc::umma(tmem + s * 64, tc::smem_desc(vl + k * 4096, 2048, 128, tc::LAYOUT_NONE), bd, IDESC, 1u);
-        }
-        tc::umma_commit(&mma_done[s]);
-        return true;
-    };
 
     if (warp == 4 * XQ) {
         // ---- one thread issues each block's MMAs as soon as its tiles have landed; it only ever
-        // waits for data --------------------------------------------------------------------------
+        // waits for data (and, at the first column block of a tile, for the tile's v) -------------
         if (lane == 0) {
-            for (int32_t j = 0; j < nblk; ++j) {
-                if (*failed || !issue_mma(j)) { *failed = 1; break; }
+            int32_t i = 0, piece = 0;
+            bool ok = true;
+            for (int64_t g = g0; g < g1 && ok; ++piece) {
+                const int32_t t = (int32_t)(g / nblk), j0 = (int32_t)(g % nblk);
+                const int32_t len = (int32_t)min((int64_t)(nblk - j0), g1 - g);
+                const LongTile lt = long_tile(P, t);
+                ok = lt.ok && tc::mbar_wait(v_ready, (uint32_t)piece & 1u);
+                tc::tc_fence_after();
+                const int32_t ksteps = (lt.rank + 15) >> 4;
+                const uint32_t vh = tc::smem_u32(Vh), vl = tc::smem_u32(Vl);
+                for (int32_t j = 0; j < len && ok; ++j, ++i) {
+                    const int s = i % S;
+                    ok = !*failed && tc::mbar_wait(&full[s], (uint32_t)(i / S) & 1u);
+                    if (!ok) break;
+                    tc::tc_fence_after();
+                    const uint32_t ba = tc::smem_u32(stages + s * C::STAGE + XT_BYTES);
+                    for (int32_t k = 0; k < ksteps; ++k) {
+                        // v: two rank groups per step, 2048 bytes apart; B tile: 16 rank rows = 2048 bytes per step
+                        const uint64_t bd = tc::smem_desc(ba + k * 2048, 16, 1024, tc::LAYOUT_SW128);
+                        tc::umma(tmem + s * 64, tc::smem_desc(vh + k * 4096, 2048, 128, tc::LAYOUT_NONE), bd, IDESC,
+                                 k > 0 ? 1u : 0u);
+                        tc::umma(tmem + s * 64, tc::smem_desc(vl + k * 4096, 2048, 128, tc::LAYOUT_NONE), bd, IDESC, 1u);
+                    }
+                    tc::umma_commit(&mma_done[s]);
+                }
+                g += len;
             }
+            if (!ok) *failed = 1;
         }
         __syncwarp();
     } else if (warp == 4 * XQ + 1) {
@@ -579,19 +551,46 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
         // store has read the stage and requests the block that reuses it.  Every stage that is not
         // being finished or stored therefore has a load in flight. ---------------------------------
         if (lane == 0) {
+            const int32_t n = (int32_t)(g1 - g0);
             int32_t issued = 0;
-            for (int32_t j = 0; j < nblk && j < S; ++j, ++issued) issue_load(j);
-            for (int32_t j = 0; j < nblk; ++j) {
+            bool ok = true;
+            // cursor of the requests (runs S blocks ahead of the cursor of the stores)
+            int32_t lt_t = (int32_t)(g0 / nblk), lj = (int32_t)(g0 % nblk);
+            LongTile llt = long_tile(P, lt_t);
+            auto issue_load = [&]() {
+                const int s = issued % S;
+                unsigned char *st = stages + s * C::STAGE;
+                tc::mbar_expect_tx(&full[s], XT_BYTES + C::BT_BYTES);
+                tc::tma_load_2d(st, &map_yb, lj * 64, llt.t0, &full[s]);
+                tc::tma_load_3d(st + XT_BYTES, &map_b, lj * 64, 0, llt.slot, &full[s]);
+                ++issued;
+                if (++lj == nblk && issued < n) {
+                    lj = 0;
+                    llt = long_tile(P, ++lt_t);
+                }
+            };
+            ok = llt.ok;
+            while (ok && issued < n && issued < S) {
+                issue_load();
+                ok = llt.ok;
+            }
+            int32_t st_t = (int32_t)(g0 / nblk), sj = (int32_t)(g0 % nblk);
+            LongTile slt = long_tile(P, st_t);
+            for (int32_t j = 0; j < n && ok; ++j) {
                 const int s = j % S;
                 if (!tc::mbar_wait(&epi_done[s], (uint32_t)(j / S) & 1u) || *failed) { ok = false; break; }
-                if (lt.rows == TC_ROWS) {
-                    tc::tma_store_2d(&map_y, (b0 + j) * 64, lt.t0, stages + s * C::STAGE);
+                if (slt.rows == TC_ROWS) {
+                    tc::tma_store_2d(&map_y, sj * 64, slt.t0, stages + s * C::STAGE);
                     tc::bulk_commit();
                     tc::bulk_wait_read<0>();
                 }
-                if (j + S < nblk) {
-                    issue_load(j + S);
-                    ++issued;
+                if (issued < n) {
+                    issue_load();
+                    ok = llt.ok;
+                }
+                if (++sj == nblk && j + 1 < n) {
+                    sj = 0;
+                    slt = long_tile(P, ++st_t);
                 }
             }
             tc::bulk_wait_read<0>();
@@ -605,65 +604,108 @@ tc_expand_kernel(const TcParams P, const __grid_constant__ CUtensorMap map_b,
         }
         __syncwarp();
     } else {
-        // ---- epilogue warps: XQ per quarter of the rows (a warp reads the tensor-memory lanes of
-        // its number modulo four), each taking 64 / XQ of the block's columns; the y_base tile
-        // (128-byte swizzle) is updated in place
+        // ---- epilogue warps: thread = row.  At the first column block of a tile they build v; per
+        // column block the y_base tile (128-byte swizzle) is updated in place -----------------------
         const int quarter = warp & 3, part = warp >> 2;
         const int m = quarter * 32 + lane;
-        for (int32_t j = 0; j < nblk; ++j) {
-            const int s = j % S;
-            // all eight warps take the same decision (a thread that left alone would strand the
-            // others at the named barrier below)
-            const uint32_t bad = (*failed != 0 || !tc::mbar_wait(&mma_done[s], (uint32_t)(j / S) & 1u)) ? 1u : 0u;
-            uint32_t any_bad;
-            asm volatile(
-                "{\n\t.reg .pred p, q;\n\t"
-                "setp.ne.u32 p, %1, 0;\n\t"
-                "bar.red.or.pred q, 1, %2, p;\n\t"
-                "selp.u32 %0, 1, 0, q;\n\t}"
-                : "=r"(any_bad)
-                : "r"(bad), "n"(XQ * TC_ROWS)
-                : "memory");
-            if (any_bad) { ok = false; *failed = 1; break; }
-            tc::tc_fence_after();
-            unsigned char *tile = stages + s * C::STAGE;
+        int32_t i = 0, piece = 0;
+        bool ok = true;
+        for (int64_t g = g0; g < g1 && ok; ++piece) {
+            const int32_t t = (int32_t)(g / nblk), j0 = (int32_t)(g % nblk);
+            const int32_t len = (int32_t)min((int64_t)(nblk - j0), g1 - g);
+            const LongTile lt = long_tile(P, t);
+            // v = sum of the tile's pieces (in order).  Stored as bf16 high and low parts in the
+            // no-swizzle K-major layout: 8 x 8 core matrices of 128 bytes, the core matrix of row
+            // group mg and rank group kg at (kg * 16 + mg) * 128 bytes.  The MMAs of the tile
+            // before have completed: this thread has waited for the last of them.
+            if (part == 0) {
+                const int32_t n_pieces = last_block_of(sp, t) - first_block_of(sp, t) + 1;
+                const float *src = P.ws + ((int64_t)lt.row0 + m) * P.RS;
+                const int64_t ks_stride = (int64_t)P.T * P.RS;
 #pragma unroll
-            for (int cc = 0; cc < 64 / XQ; cc += 16) {
-                const int c = part * (64 / XQ) + cc;
-                uint32_t r[16];
-                tc::tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + s * 64 + c, r);
-                tc::tmem_ld_wait();
+                for (int kg = 0; kg < RP / 8; ++kg) {
+                    float v[8];
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int chunk = (c >> 3) + h;
-                    uint4 *p = reinterpret_cast<uint4 *>(tile + m * 128 + ((chunk ^ (m & 7)) << 4));
-                    float acc[8];
+                    for (int e = 0; e < 8; ++e) v[e] = 0.0f;
+                    for (int32_t q = 0; q < n_pieces && lt.ok && m < lt.rows; ++q) {   // rows past a short tile's end stay zero
+                        const float4 a = *reinterpret_cast<const float4 *>(src + q * ks_stride + kg * 8);
+                        const float4 b = *reinterpret_cast<const float4 *>(src + q * ks_stride + kg * 8 + 4);
+                        v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
+                        v[4] += b.x; v[5] += b.y; v[6] += b.z; v[7] += b.w;
+                    }
+                    uint32_t hi[4], lo[4];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) acc[e] = __uint_as_float(r[h * 8 + e]);
-                    *p = finish8(acc, *p, lt.scale);
+                    for (int e = 0; e < 8; e += 2) {
+                        const float v0 = kg * 8 + e < lt.rank ? v[e] : 0.0f;
+                        const float v1 = kg * 8 + e + 1 < lt.rank ? v[e + 1] : 0.0f;
+                        const __nv_bfloat16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
+                        hi[e / 2] = pack2(__bfloat162float(h0), __bfloat162float(h1));
+                        lo[e / 2] = pack2(v0 - __bfloat162float(h0), v1 - __bfloat162float(h1));
+                    }
+                    const int off = (kg * 16 + (m >> 3)) * 128 + (m & 7) * 16;
+                    *reinterpret_cast<uint4 *>(Vh + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<uint4 *>(Vl + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                 }
+                tc::fence_proxy_async();     // v was written with ordinary stores and is read by the MMA unit
             }
-            tc::tc_fence_before();
-            if (lt.rows < TC_ROWS) {
-                // short tile: the rows after it belong to other tokens, so each thread stores its own row
-                const int32_t colb = (b0 + j) * 64;
-                if (m < lt.rows) {
-                    __nv_bfloat16 *yrow = P.y + (int64_t)(lt.t0 + m) * P.ldy + colb;
+            tc::mbar_arrive(v_ready);
+            for (int32_t j = 0; j < len; ++j, ++i) {
+                const int s = i % S;
+                // all four warps take the same decision (a thread that left alone would strand the
+                // others at the named barrier)
+                const uint32_t bad =
+                    (*failed != 0 || !lt.ok || !tc::mbar_wait(&mma_done[s], (uint32_t)(i / S) & 1u)) ? 1u : 0u;
+                uint32_t any_bad;
+                asm volatile(
+                    "{\n\t.reg .pred p, q;\n\t"
+                    "setp.ne.u32 p, %1, 0;\n\t"
+                    "bar.red.or.pred q, 1, %2, p;\n\t"
+                    "selp.u32 %0, 1, 0, q;\n\t}"
+                    : "=r"(any_bad)
+                    : "r"(bad), "n"(XQ * TC_ROWS)
+                    : "memory");
+                if (any_bad) { ok = false; *failed = 1; break; }
+                tc::tc_fence_after();
+                unsigned char *tile = stages + s * C::STAGE;
 #pragma unroll
-                    for (int chunk = part * (8 / XQ); chunk < (part + 1) * (8 / XQ); ++chunk)
-                        if (colb + chunk * 8 < P.tv.d_out)
-                            *reinterpret_cast<uint4 *>(yrow + chunk * 8) =
-                                *reinterpret_cast<const uint4 *>(tile + m * 128 + ((chunk ^ (m & 7)) << 4));
+                for (int cc = 0; cc < 64 / XQ; cc += 16) {
+                    const int c = part * (64 / XQ) + cc;
+                    uint32_t r[16];
+                    tc::tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + s * 64 + c, r);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int chunk = (c >> 3) + h;
+                        uint4 *p = reinterpret_cast<uint4 *>(tile + m * 128 + ((chunk ^ (m & 7)) << 4));
+                        float acc[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[e] = __uint_as_float(r[h * 8 + e]);
+                        *p = finish8(acc, *p, lt.scale);
+                    }
                 }
-            } else {
-                tc::fence_proxy_async();    // the tile is read by the TMA store
+                tc::tc_fence_before();
+                if (lt.rows < TC_ROWS) {
+                    // short tile: the rows after it belong to other tokens, so each thread stores its own row
+                    const int32_t colb = (j0 + j) * 64;
+                    if (m < lt.rows) {
+                        __nv_bfloat16 *yrow = P.y + (int64_t)(lt.t0 + m) * P.ldy + colb;
+#pragma unroll
+                        for (int chunk = part * (8 / XQ); chunk < (part + 1) * (8 / XQ); ++chunk)
+                            if (colb + chunk * 8 < P.tv.d_out)
+                                *reinterpret_cast<uint4 *>(yrow + chunk * 8) =
+                                    *reinterpret_cast<const uint4 *>(tile + m * 128 + ((chunk ^ (m & 7)) << 4));
+                    }
+                } else {
+                    tc::fence_proxy_async();    // the tile is read by the TMA store
+                }
+                tc::mbar_arrive(&epi_done[s]);  // 128 arrivals: every row of the stage is finished
             }
-            tc::mbar_arrive(&epi_done[s]);  // every epilogue thread: all rows and columns of the stage are finished
+            g += len;
         }
     }
-    if (tid == 0 && *failed) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
     tc::tc_fence_before();
     __syncthreads();
+    if (tid == 0 && *failed) atomicAdd(&P.pool.status[STATUS_TIMEOUTS], 1);
     if (warp == 4 * XQ) tc::tmem_dealloc(tmem, C::TMEM_COLS);
 }
 
@@ -717,7 +759,7 @@ static bool make_map_3d(CUtensorMap *m, const void *base, int64_t d, int64_t r_m
 
 template <int RP>
 static lora_status_t launch_tc_bucket(lora_pool_t *pool, const TcParams &P, const ApplyParams &AP,
-                                      int32_t units, cudaStream_t stream) {
+                                      cudaStream_t stream) {
     CUtensorMap mx, myb, my, ma, mb;
     const __nv_bfloat16 *w = pool->weights_dev;
     if (!make_map_2d(&mx, AP.x, AP.T, AP.tv.d_in, AP.ldx) || !make_map_2d(&myb, AP.yb, AP.T, AP.tv.d_out, AP.ldyb) ||
@@ -738,7 +780,7 @@ static lora_status_t launch_tc_bucket(lora_pool_t *pool, const TcParams &P, cons
     tc_shrink_kernel<RP><<<P.shrink_grid, TCS_THREADS, SH_SMEM, stream>>>(P, mx, ma);
     lora_status_t s = count_launch();
     if (s != LORA_OK) return s;
-    tc_expand_kernel<RP><<<dim3(units, P.NS), TCX_THREADS, ExpandCfg<RP>::SMEM, stream>>>(P, mb, myb, my);
+    tc_expand_kernel<RP><<<P.expand_grid, TCX_THREADS, ExpandCfg<RP>::SMEM, stream>>>(P, mb, myb, my);
     return count_launch();
 }
 
@@ -779,18 +821,10 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
         (AP.ldy % 8))
         return LORA_OK;
     const int32_t RS = rank_bucket(pool->r_max) < 16 ? 16 : rank_bucket(pool->r_max);
-    const int32_t max_long = (AP.T + TC_MIN_ROWS - 1) / TC_MIN_ROWS < AP.T / TC_ROWS + AP.meta_slots
-                                 ? (AP.T + TC_MIN_ROWS - 1) / TC_MIN_ROWS
-                                 : AP.T / TC_ROWS + AP.meta_slots;   // bound on tiles this path takes
     if (!pool->meta_has_list(AP.meta)) return LORA_OK;   // built before the batch qualified (tuning changed)
     const size_t per_split = (size_t)AP.T * RS * sizeof(float);
     if (!workspace || workspace_bytes < per_split || ((uintptr_t)workspace & 15)) return LORA_OK;
     int32_t KS = (int32_t)(workspace_bytes / per_split < 8 ? workspace_bytes / per_split : 8);   // slabs of partials
-    int32_t NS = (4 * pool->sm_count + max_long - 1) / max_long;
-    if (pool->tuning[8] > 0) NS = pool->tuning[8];   // tuning key 8: column splits of a tile in the expand
-    const int32_t nblk = (AP.tv.d_out + 63) / 64;
-    if (NS > nblk) NS = nblk;
-    if (NS < 1) NS = 1;
 
     TcParams P;
     P.pool = AP.pool;
@@ -800,7 +834,6 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
     P.T = AP.T;
     P.RS = RS;
     P.KS = KS;
-    P.NS = NS;
     const MetaLayout L = meta_layout(AP.T, AP.meta_slots, AP.tile_m);
     if (L.words > 0x7fffffff) return LORA_OK;
     P.moff_perm = (int32_t)L.perm;
@@ -809,19 +842,23 @@ lora_status_t launch_tc_long_tiles(lora_pool_t *pool, const ApplyParams &AP, voi
     P.list = const_cast<int32_t *>(AP.meta) + L.long_list;
     P.list_cap = L.cap_tile;
     P.shrink_grid = 2 * pool->sm_count;   // two blocks fit on an SM: the grid fills the GPU exactly once
+    // The expand's walk is cut finer: four waves of blocks (two per SM at a time), so that blocks that
+    // start late or share their SM with the fused kernel do not leave the others waiting at the end
+    // (blocks per SM in the grid 2 / 4 / 8 / 12 / 16: prefill step 577 / 545 / 540 / 553 / 566 us).
+    // Tuning key 8 overrides the number of blocks per SM.
+    P.expand_grid = (pool->tuning[8] > 0 ? pool->tuning[8] : 8) * pool->sm_count;
     if (check_only) {   // nothing has been launched: the caller only asks whether the path applies
         *handled = true;
         return LORA_OK;
     }
-    const int32_t units = max_long;   // block columns of the expand: one per list entry, the unused ones leave at once
 
     P.y = AP.y;
     P.ldy = AP.ldy;
     // one pair of launches for every rank: the kernels are sized for the pool's largest rank
     // bucket, and the rows above a slot's rank are zero
-    lora_status_t s = RS <= 16   ? launch_tc_bucket<16>(pool, P, AP, units, stream)
-                      : RS == 32 ? launch_tc_bucket<32>(pool, P, AP, units, stream)
-                                 : launch_tc_bucket<64>(pool, P, AP, units, stream);
+    lora_status_t s = RS <= 16   ? launch_tc_bucket<16>(pool, P, AP, stream)
+                      : RS == 32 ? launch_tc_bucket<32>(pool, P, AP, stream)
+                                 : launch_tc_bucket<64>(pool, P, AP, stream);
     if (s == LORA_OK) *handled = true;
     return s;
 }
